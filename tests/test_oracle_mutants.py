@@ -1,0 +1,80 @@
+"""The pins have teeth: a mistake planted in a copy of the reference makes at least one fail.
+
+Each mutant is the reference's C source with one line changed (a flipped sign, a dropped
+term, a wrong index, another reading of the staleness).  It is built in a temporary folder
+and the pin tests are re-run against it; every mutant must be caught.
+"""
+import json
+import os
+import shutil
+import subprocess
+
+import pytest
+
+from oracle import reference as R
+from tests import test_oracle_arrivals as TA
+from tests import test_oracle_update as TU
+
+ORACLE_DIR = os.path.dirname(os.path.abspath(R.__file__))
+
+MUTANTS = {
+    "decay_sign": ("update_rule.inc", "const REAL t = acc + d * w[k];", "const REAL t = acc - d * w[k];"),
+    "descent_sign": ("update_rule.inc", "w[k] = w[k] - v[k];", "w[k] = w[k] + v[k];"),
+    "momentum_dropped": ("update_rule.inc", "v[k] = m * v[k] + t;", "v[k] = t;"),
+    "decay_dropped": ("update_rule.inc", "const REAL t = acc + d * w[k];", "const REAL t = acc;"),
+    "no_averaging": ("update_rule.inc", "((double)c * (double)sigma[l])", "((double)sigma[l])"),
+    "wrong_gradient_index": ("update_rule.inc", "acc = acc + s[l] * grads[l][k];", "acc = acc + s[l] * grads[0][k];"),
+    "wrong_scale_index": ("update_rule.inc", "acc = acc + s[l] * grads[l][k];", "acc = acc + s[0] * grads[l][k];"),
+    "decay_unmodulated": ("update_rule.inc", "const REAL d = ROUND_SCALE(wd * S);", "const REAL d = ROUND_SCALE(wd * alpha0);"),
+    "staleness_plus_one": ("softsync_oracle.c", "sigma = tau > 0 ? tau : 1;", "sigma = tau + 1;"),
+    "staleness_ignored": ("softsync_oracle.c", "sigma = tau > 0 ? tau : 1;", "sigma = 1;"),
+    "clock_jumps": ("softsync_oracle.c", "ps->ts += 1;", "ps->ts += ps->c;"),
+    "arrival_order_sum": ("softsync_oracle.c", "if (a->learner != b->learner) return a->learner < b->learner;\n    return a->push_index < b->push_index;", "(void)a; (void)b; return 0;"),
+    "group_one_short": ("softsync_oracle.c", "if (ps->npending == ps->c) { apply_pending(ps); return 1; }",
+                        "if (ps->npending == ps->c || (ps->c > 1 && ps->npending == ps->c - 1)) { ps->c = ps->npending; apply_pending(ps); return 1; }"),
+    "stale_pull": ("softsync_oracle.c", "ps->pulled_ts[learner] = ps->ts;", "ps->pulled_ts[learner] = ps->ts > 0 ? ps->ts - 1 : 0;"),
+}
+
+
+def _pins():
+    examples = json.load(open(TU.GOLDEN))["examples"]
+    pins = [lambda e=e, p=p: TU.test_hand_worked_examples_exact(e, p) for e in examples for p in (32, 64)]
+    pins += [
+        TU.test_single_learner_is_sequential_momentum_sgd_bit_for_bit,
+        TU.test_single_learner_matches_library_sgd_optimizer,
+        lambda: TU.test_one_softsync_with_barrier_is_synchronous_averaged_sgd(4),
+        TU.test_downpour_case_is_per_push_sgd,
+        lambda: TU.test_plain_rule_is_a_weighted_sum_of_gradients("exp", 12, 3),
+        TU.test_momentum_is_a_geometric_sum_of_past_steps,
+        TU.test_decay_and_momentum_follow_the_linear_recurrence_in_matrix_form,
+        TU.test_arrival_order_inside_a_group_does_not_change_the_bits,
+        lambda: TA.test_clock_and_staleness_against_brute_force_recount("uniform", 18, 4),
+        lambda: TA.test_homogeneous_learners_match_measured_staleness(1, 0.8, 1.2),
+    ]
+    return pins
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_planted_mistake_is_caught(name, tmp_path):
+    fname, old, new = MUTANTS[name]
+    for f in ("softsync_oracle.c", "arrival_sim.c", "update_rule.inc"):
+        shutil.copy(os.path.join(ORACLE_DIR, f), tmp_path / f)
+    src = (tmp_path / fname).read_text()
+    assert src.count(old) == 1, "mutation site must exist exactly once"
+    (tmp_path / fname).write_text(src.replace(old, new))
+    so = str(tmp_path / ("mutant_%s.so" % name))
+    subprocess.run(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fPIC", "-shared", "-o", so,
+                    "softsync_oracle.c", "arrival_sim.c", "-lm"], check=True, cwd=tmp_path)
+    caught = 0
+    with R.use_library(so):
+        for pin in _pins():
+            try:
+                pin()
+            except (AssertionError, ValueError):
+                caught += 1
+    assert caught >= 1, "no pin noticed the planted mistake %r" % name
+
+
+def test_unmutated_reference_passes_the_same_pins():
+    for pin in _pins():
+        pin()

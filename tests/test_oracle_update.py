@@ -1,0 +1,303 @@
+"""Pins for the reference's update arithmetic (everything here runs on the CPU).
+
+Each test compares the reference with something that is fixed outside it:
+hand-worked numbers (tests/golden), a library optimiser, a closed form, or a
+special case in which the method collapses to a textbook rule.
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import reference as R
+from tests.helpers import replay_reference, staleness_by_recount, rel_l2
+from workloads import generators as G
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "worked_softsync.json")
+MODS = {"inv_staleness": R.MOD_INV_STALENESS, "constant": R.MOD_CONSTANT}
+
+
+def _grads(seed, lam, pushes_per_learner, n, std=1e-3, dtype=torch.float32):
+    return {(l, p): G.gradient(seed, l, p, n, std, dtype=dtype) for l in range(lam) for p in range(pushes_per_learner)}
+
+
+# ---------------------------------------------------------------- hand-worked examples
+@pytest.mark.parametrize("precision", [32, 64])
+@pytest.mark.parametrize("example", json.load(open(GOLDEN))["examples"], ids=lambda e: e["name"])
+def test_hand_worked_examples_exact(example, precision):
+    ex = example
+    ps = R.ReferencePS(len(ex["w0"]), ex["num_learners"], ex["n"], ex["alpha0"], ex["momentum"],
+                       ex["weight_decay"], MODS[ex["modulation"]], precision)
+    ps.set_weights(np.asarray(ex["w0"], np.float32))
+    done = 0
+    for ev in ex["events"]:
+        if ev[0] == "pull":
+            ps.pull(ev[1])
+            continue
+        fired = ps.push(ev[1], np.asarray(ev[2], np.float32))
+        if fired:
+            exp = ex["updates"][done]
+            done += 1
+            w, v = ps.state()
+            assert w.tolist() == exp["w"] and v.tolist() == exp["v"]
+            assert ps.timestamp == exp["ts"]
+            rows = ps.log()[-len(exp["members"]):]
+            got = [[int(r["learner"]), int(r["push_index"]), int(r["ts_grad"]), int(r["tau"]),
+                    int(r["sigma"]), float(r["scale"])] for r in rows]
+            assert got == exp["members"]
+            assert all(float(r["decay"]) == exp["decay"] for r in rows)
+    assert done == len(ex["updates"])
+
+
+# ---------------------------------------------------------------- collapses to textbook rules
+def test_single_learner_is_sequential_momentum_sgd_bit_for_bit():
+    """lambda = 1, n = 1: every gradient has tau = 0 and the method is plain momentum SGD."""
+    n, steps = 257, 40
+    a, m, wd = np.float32(0.01), np.float32(0.9), np.float32(5e-4)
+    w0 = G.normal_like(G.stream_key(1, G.STREAM_WEIGHTS), 0, n, 0.01).numpy()
+    ps = R.ReferencePS(n, 1, 1, float(a), float(m), float(wd), R.MOD_INV_STALENESS, 32)
+    ps.set_weights(w0)
+    w, v = w0.copy(), np.zeros(n, np.float32)
+    awd = np.float32(np.float64(wd) * np.float64(a))
+    for p in range(steps):
+        g = G.gradient(1, 0, p, n, 1e-3).numpy()
+        ps.pull(0)
+        assert ps.push(0, g)
+        v = m * v + (a * g + awd * w)          # textbook: v <- m v + lr (g + wd w); w <- w - v
+        w = w - v
+    wr, vr = ps.state()
+    assert np.array_equal(wr.astype(np.float32), w) and np.array_equal(vr.astype(np.float32), v)
+    assert ps.timestamp == steps
+    assert (ps.log()["sigma"] == 1).all()
+
+
+def test_single_learner_matches_library_sgd_optimizer():
+    """Same special case against torch.optim.SGD (lr outside the velocity: v_here = lr * buf)."""
+    n, steps = 64, 60
+    lr, m, wd = 0.01, 0.9, 5e-4
+    w0 = G.normal_like(G.stream_key(2, G.STREAM_WEIGHTS), 0, n, 0.01)
+    ps = R.ReferencePS(n, 1, 1, lr, m, wd, R.MOD_INV_STALENESS, 64)
+    ps.set_weights(w0.numpy())
+    p = torch.nn.Parameter(w0.double().clone())
+    f32 = lambda x: float(np.float32(x))
+    opt = torch.optim.SGD([p], lr=f32(lr), momentum=f32(m), weight_decay=f32(wd))
+    for s in range(steps):
+        g = G.gradient(2, 0, s, n, 1e-3)
+        ps.pull(0)
+        ps.push(0, g.numpy())
+        p.grad = g.double()
+        opt.step()
+    w, v = ps.state()
+    assert rel_l2(w, p.detach().numpy()) < 1e-13
+    buf = opt.state[p]["momentum_buffer"].numpy()
+    assert rel_l2(v, f32(lr) * buf) < 1e-12
+
+
+@pytest.mark.parametrize("lam", [2, 4, 5])
+def test_one_softsync_with_barrier_is_synchronous_averaged_sgd(lam):
+    """n = 1 and everybody pulls after the update: tau = 0, Eq. 2 becomes Eq. 1 (hardsync),
+    i.e. SGD on the mean of the lambda gradients; with momentum and decay that is library SGD."""
+    n, rounds = 48, 25
+    lr, m, wd = 0.05, 0.9, 5e-4
+    w0 = G.normal_like(G.stream_key(3, G.STREAM_WEIGHTS), 0, n, 0.01)
+    f32 = lambda x: float(np.float32(x))
+    for momentum, decay in ((0.0, 0.0), (m, wd)):
+        ps = R.ReferencePS(n, lam, 1, lr, momentum, decay, R.MOD_INV_STALENESS, 64)
+        ps.set_weights(w0.numpy())
+        p = torch.nn.Parameter(w0.double().clone())
+        opt = torch.optim.SGD([p], lr=f32(lr), momentum=f32(momentum), weight_decay=f32(decay))
+        plain = w0.double().numpy().copy()
+        for r in range(rounds):
+            for l in range(lam):
+                ps.pull(l)
+            gs = [G.gradient(3, l, r, n, 1e-3).double() for l in range(lam)]
+            order = np.random.default_rng(r).permutation(lam)
+            for l in order:
+                fired = ps.push(int(l), gs[l].float().numpy())
+            assert fired
+            p.grad = torch.stack(gs).mean(0)
+            opt.step()
+            plain = plain - f32(lr) * np.mean(np.stack([g.numpy() for g in gs]), axis=0)   # Eq. 1
+        w, _ = ps.state()
+        assert (ps.log()["tau"] == 0).all()
+        assert rel_l2(w, p.detach().numpy()) < 1e-12
+        if momentum == 0.0 and decay == 0.0:
+            assert rel_l2(w, plain) < 1e-12
+    # the fp32 reference agrees with the fp64 one to fp32 rounding
+    ps32 = R.ReferencePS(n, lam, 1, lr, m, wd, R.MOD_INV_STALENESS, 32)
+    ps32.set_weights(w0.numpy())
+    for r in range(rounds):
+        for l in range(lam):
+            ps32.pull(l)
+        for l in range(lam):
+            ps32.push(l, G.gradient(3, l, r, n, 1e-3).numpy())
+    assert rel_l2(ps32.state()[0], p.detach().numpy()) < 1e-6
+
+
+def test_downpour_case_is_per_push_sgd():
+    """n = lambda with a constant rate is Downpour SGD: theta <- theta - alpha0 * dtheta per push."""
+    lam, n_el, pushes = 6, 32, 120
+    a0 = float(np.float32(0.02))
+    k, l = R.simulate_arrivals("exp", lam, pushes, 9)
+    ps = R.ReferencePS(n_el, lam, lam, a0, 0.0, 0.0, R.MOD_CONSTANT, 64)
+    w0 = G.normal_like(G.stream_key(4, G.STREAM_WEIGHTS), 0, n_el, 0.01).numpy()
+    ps.set_weights(w0)
+    total = np.zeros(n_el)
+    def grad(a, b):
+        g = G.gradient(4, a, b, n_el, 1e-3).numpy()
+        total[:] += g.astype(np.float64)
+        return g
+    replay_reference(ps, k, l, grad)
+    assert ps.timestamp == pushes
+    assert rel_l2(ps.state()[0], w0.astype(np.float64) - a0 * total) < 1e-13
+
+
+# ---------------------------------------------------------------- closed forms
+@pytest.mark.parametrize("model,lam,n", [("exp", 8, 8), ("exp", 12, 3), ("uniform", 18, 4), ("lognormal", 10, 5)])
+def test_plain_rule_is_a_weighted_sum_of_gradients(model, lam, n):
+    """m = 0, wd = 0: theta_K = theta_0 - sum over pushes of alpha0/(c max(tau,1)) * dtheta
+    (Eq. 2 summed over updates, Eq. 3), with tau recounted from the raw trace."""
+    n_el, pushes = 40, 240
+    c = lam // n
+    a0 = float(np.float32(0.03))
+    k, l = R.simulate_arrivals(model, lam, pushes, 17)
+    tau, _ = staleness_by_recount(k, l, c)
+    ps = R.ReferencePS(n_el, lam, n, a0, 0.0, 0.0, R.MOD_INV_STALENESS, 64)
+    w0 = G.normal_like(G.stream_key(5, G.STREAM_WEIGHTS), 0, n_el, 0.01).numpy()
+    ps.set_weights(w0)
+    seen = []
+    def grad(a, b):
+        g = G.gradient(5, a, b, n_el, 1e-3).numpy()
+        seen.append(g.astype(np.float64))
+        return g
+    replay_reference(ps, k, l, grad)
+    used = (pushes // c) * c
+    weights = a0 / (c * np.maximum(tau[:used], 1))
+    expect = w0.astype(np.float64) - np.einsum("p,pk->k", weights, np.stack(seen[:used]))
+    assert rel_l2(ps.state()[0], expect) < 1e-13
+    assert tau.max() >= 2       # the case really exercises staleness
+
+
+def test_momentum_is_a_geometric_sum_of_past_steps():
+    """wd = 0: v_K = sum_i m^(K-1-i) u_i and theta_K = theta_0 - sum_i u_i (1 - m^(K-i))/(1 - m),
+    where u_i is the Eq. 2 step of update i."""
+    lam, n, n_el, pushes = 6, 2, 16, 90
+    c = lam // n
+    a0, m = float(np.float32(0.02)), float(np.float32(0.9))
+    k, l = R.simulate_arrivals("exp", lam, pushes, 23)
+    tau, _ = staleness_by_recount(k, l, c)
+    ps = R.ReferencePS(n_el, lam, n, a0, m, 0.0, R.MOD_INV_STALENESS, 64)
+    w0 = np.zeros(n_el, np.float32)
+    ps.set_weights(w0)
+    seen = []
+    def grad(a, b):
+        g = G.gradient(6, a, b, n_el, 1e-3).numpy()
+        seen.append(g.astype(np.float64))
+        return g
+    replay_reference(ps, k, l, grad)
+    K = pushes // c
+    scaled = (a0 / (c * np.maximum(tau[:K * c], 1)))[:, None] * np.stack(seen[:K * c])
+    u = scaled.reshape(K, c, n_el).sum(1)
+    i = np.arange(K)
+    v_expect = ((m ** (K - 1 - i))[:, None] * u).sum(0)
+    w_expect = -(((1 - m ** (K - i)) / (1 - m))[:, None] * u).sum(0)
+    w, v = ps.state()
+    assert rel_l2(v, v_expect) < 1e-12 and rel_l2(w, w_expect) < 1e-12
+
+
+def test_decay_and_momentum_follow_the_linear_recurrence_in_matrix_form():
+    """Per element the update is x <- A_i x + b_i with x = (w, v),
+    A_i = [[1 - d_i, -m], [d_i, m]], b_i = (-u_i, u_i), d_i = wd * sum_l s_l.
+    Checked with an accumulated matrix product instead of stepping the scalars."""
+    lam, n, pushes = 9, 3, 150
+    c = lam // n
+    a0, m, wd = float(np.float32(0.05)), float(np.float32(0.8)), float(np.float32(0.01))
+    k, l = R.simulate_arrivals("lognormal", lam, pushes, 31)
+    tau, _ = staleness_by_recount(k, l, c)
+    ps = R.ReferencePS(1, lam, n, a0, m, wd, R.MOD_INV_STALENESS, 64)
+    w0 = np.array([0.5], np.float32)
+    ps.set_weights(w0)
+    seen = []
+    def grad(a, b):
+        g = G.gradient(7, a, b, 1, 1e-2).numpy()
+        seen.append(float(g[0]))
+        return g
+    replay_reference(ps, k, l, grad)
+    K = pushes // c
+    s = (a0 / (c * np.maximum(tau[:K * c], 1))).reshape(K, c)
+    u = (s * np.asarray(seen[:K * c]).reshape(K, c)).sum(1)
+    d = wd * s.sum(1)
+    # homogeneous coordinates: one 3x3 affine map per update, multiplied up
+    M = np.eye(3)
+    for i in range(K):
+        step = np.array([[1 - d[i], -m, -u[i]], [d[i], m, u[i]], [0, 0, 1]])
+        M = step @ M
+    x = M @ np.array([0.5, 0.0, 1.0])
+    w, v = ps.state()
+    assert abs(w[0] - x[0]) < 1e-12 * max(1, abs(x[0])) and abs(v[0] - x[1]) < 1e-12
+    assert tau.max() >= 3
+
+
+# ---------------------------------------------------------------- invariants of the readings
+def test_arrival_order_inside_a_group_does_not_change_the_bits():
+    lam, n_el = 5, 33
+    w0 = G.normal_like(G.stream_key(8, G.STREAM_WEIGHTS), 0, n_el, 0.01).numpy()
+    results = []
+    for perm_seed in range(4):
+        ps = R.ReferencePS(n_el, lam, 1, 0.01, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+        ps.set_weights(w0)
+        for r in range(6):
+            for l in range(lam):
+                ps.pull(l)
+            for l in np.random.default_rng(perm_seed * 100 + r).permutation(lam):
+                ps.push(int(l), G.gradient(8, int(l), r, n_el, 1e-3).numpy())
+        results.append(ps.state())
+    for w, v in results[1:]:
+        assert np.array_equal(w, results[0][0]) and np.array_equal(v, results[0][1])
+
+
+def test_bf16_gradients_are_widened_exactly():
+    n_el, lam = 64, 3
+    w0 = G.normal_like(G.stream_key(9, G.STREAM_WEIGHTS), 0, n_el, 0.01).numpy()
+    a = R.ReferencePS(n_el, lam, 3, 0.01, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    b = R.ReferencePS(n_el, lam, 3, 0.01, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    a.set_weights(w0); b.set_weights(w0)
+    for l in range(lam):
+        a.pull(l); b.pull(l)
+    for p in range(5):
+        for l in range(lam):
+            g = G.gradient(9, l, p, n_el, 1e-4, dtype=torch.bfloat16)
+            a.push(l, g.view(torch.int16).numpy().view(np.uint16))
+            b.push(l, g.float().numpy())
+    assert np.array_equal(a.state()[0], b.state()[0]) and np.array_equal(a.state()[1], b.state()[1])
+    assert a.timestamp == 15
+
+
+def test_fp32_reference_tracks_fp64_reference():
+    """Noise floor of keeping the state in fp32, on the small benchmark shape."""
+    from workloads import configs
+    cfg = configs.TINY_SOFTSYNC
+    n_el = 4096
+    k, l = R.simulate_arrivals(cfg.arrival_model, cfg.num_learners, 400, 1)
+    w0 = G.normal_like(G.stream_key(10, G.STREAM_WEIGHTS), 0, n_el, cfg.weight_std).numpy()
+    out = []
+    for prec in (32, 64):
+        ps = R.ReferencePS(n_el, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
+                           R.MOD_INV_STALENESS, prec)
+        ps.set_weights(w0)
+        replay_reference(ps, k, l, lambda a, b: G.gradient(10, a, b, n_el, cfg.grad_std).numpy())
+        out.append(ps.state())
+    assert rel_l2(out[0][0], out[1][0]) < 1e-6
+    assert rel_l2(out[0][1], out[1][1]) < 1e-5
+
+
+def test_rejects_bad_arguments():
+    with pytest.raises(ValueError):
+        R.ReferencePS(4, 3, 4, 0.1, 0.0, 0.0)          # n > lambda
+    ps = R.ReferencePS(4, 3, 3, 0.1, 0.0, 0.0)
+    with pytest.raises(ValueError):
+        ps.push(0, np.zeros(4, np.float32))            # push before any pull
+    with pytest.raises(ValueError):
+        ps.pull(3)

@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Throughput of the n-softsync parameter-server update on B200.
+
+A step is one pass of the whole server path for one weight update of the large-net softsync
+workload (60,965,224 fp32 parameters, lambda = 18 learners, n = 4, c = 4 fp32 gradients per
+update): the learners' timestamp pulls, c gradient pushes (timestamp check, staleness, grouping),
+the scale table, ONE fused sumGradients+applyUpdate kernel launch, and the timestamp advance.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints one JSON line.  `value` is gradient elements applied per second (c * N * K / time) with
+the gradients already resident in HBM; `e2e` is the same metric with every gradient copied from
+pinned host memory and the updated weights copied back to the host inside the timed region.
+With N > 1 (torchrun, one process per GPU) every rank runs an independent server replica: the
+path has no exchange step, so there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from workloads import arrivals, configs, generators as G
+
+METRIC = "ps_gradient_elements_per_sec"
+UNIT = "grad-elements/s"
+FALLBACK_HBM_GBS = 6650.0
+POOL_BUFFERS = 8
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(num_params: int, entries: int, grad_bytes: int) -> int:
+    """Bytes one kernel launch must move: every gradient once, theta and v read and written once."""
+    return num_params * (entries * grad_bytes + 16)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs (read-only NVML)."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:                                   # CUDA_VISIBLE_DEVICES may renumber: match by UUID
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _reason_names(self, mask: int):
+        nv = self.nv
+        table = {
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        return [k for k, bit in table.items() if mask & bit]
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.reasons.update(self._reason_names(mask))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        return False
+
+    def summary(self):
+        if self.nv is None or not self.samples:
+            return self._smi_once()
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": float(self.max_mhz),
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+    def _smi_once(self):
+        try:
+            out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=clocks.sm,clocks.max.sm",
+                                  "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=10).stdout
+            a, b = [float(x) for x in out.strip().split(",")]
+            return {"sm_mhz": a, "sm_max_mhz": b, "reasons": [], "samples": 1, "note": "sampled after the timed region"}
+        except Exception:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+
+
+def max_over_ranks(values, device, world: int):
+    """Slowest rank decides: element-wise maximum of per-rank timings (the only cross-rank exchange)."""
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(world: int, elems_per_step: int, steps: int, elapsed_ms: float) -> float:
+    """Units all ranks processed divided by the slowest rank's time."""
+    return world * elems_per_step * steps / (elapsed_ms * 1e-3)
+
+
+def step_events(cfg, num_steps: int):
+    """Per step, the list of trace events up to and including the push that completes a group."""
+    kinds, learners = arrivals.make_trace(cfg.arrival_model, cfg.num_learners, num_steps * cfg.c, cfg.seed)
+    steps, cur, pushes = [], [], 0
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        cur.append((k, l))
+        if k == arrivals.PUSH:
+            pushes += 1
+            if pushes % cfg.c == 0:
+                steps.append(cur)
+                cur = []
+    return steps
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args, cfg, rank, world, local_rank):
+    import paper_1511_05950_b200 as P
+    import torch.distributed as dist
+
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    layout = cfg.layout()
+    n = layout.num_params
+    tdt = torch.bfloat16 if cfg.grad_dtype == "bf16" else torch.float32
+    gbytes = 2 if cfg.grad_dtype == "bf16" else 4
+    fuse_t = cfg.fuse_t
+    groups_per_step = fuse_t                      # a step = one kernel pass = fuse_t updates
+
+    ps = P.ParameterServer(n, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
+                           cfg.modulation, cfg.grad_dtype, fuse_t, device=dev)
+    ps.init_weights(G.initial_weights(layout, cfg.seed + rank, cfg.weight_std, device=dev))
+    pool_n = max(POOL_BUFFERS, 2 * cfg.c * fuse_t)
+    pool = [G.gradient(cfg.seed + rank, i, 0, n, cfg.grad_std, dtype=tdt, device=dev) for i in range(pool_n)]
+    total_steps = args.warmup + args.steps
+    ev_steps = step_events(cfg, total_steps * groups_per_step)
+
+    cursor = {"i": 0}
+    pulled = {}
+
+    def one_step(events, step_index: int, grads):
+        for gi in range(groups_per_step):
+            for k, l in events[step_index * groups_per_step + gi]:
+                if k == arrivals.PULL:
+                    pulled[l] = ps.pull_weights()
+                else:
+                    g = grads[cursor["i"] % len(grads)]
+                    cursor["i"] += 1
+                    ps.push_gradient(l, g, pulled[l])
+        done = ps.apply_update()
+        assert done == groups_per_step
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for s in range(args.warmup):
+        one_step(ev_steps, s, pool)
+    ps.synchronize()
+    ps.set_option(P.PS_OPT_TIMING, 1)
+    ps.kernel_time()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        start.record()
+        for s in range(args.warmup, total_steps):
+            one_step(ev_steps, s, pool)
+        stop.record()
+        torch.cuda.synchronize(dev)
+    barrier()
+    elapsed_ms = start.elapsed_time(stop)
+    kernel_ms, launches = ps.kernel_time()
+    ps.set_option(P.PS_OPT_TIMING, 0)
+    assert launches == args.steps
+
+    # ---- end to end: gradients from pinned host memory, updated weights back to the host
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    host_pool = [torch.empty(n, dtype=tdt).pin_memory() for _ in range(min(4, pool_n))]
+    for hb, db in zip(host_pool, pool):
+        hb.copy_(db)
+    w_host = torch.empty(n, dtype=torch.float32).pin_memory()
+    ps.bind_staging(2 * cfg.c * fuse_t)
+    ps.init_weights(G.initial_weights(layout, cfg.seed + rank, cfg.weight_std, device=dev))
+    pulled.clear()
+    e2e_events = step_events(cfg, (1 + e2e_steps) * groups_per_step)
+
+    def e2e_step(s):
+        one_step(e2e_events, s, host_pool)
+        ps.pull_weights(w_host)                    # device -> host read of the step's result (synchronous)
+
+    e2e_step(0)
+    barrier()
+    t0 = time.perf_counter()
+    for s in range(1, 1 + e2e_steps):
+        e2e_step(s)
+    torch.cuda.synchronize(dev)
+    e2e_s = time.perf_counter() - t0
+    barrier()
+
+    elapsed_ms, e2e_ms, kern_ms = max_over_ranks([elapsed_ms, e2e_s * 1e3, kernel_ms / max(1, launches)], dev, world)
+
+    elems_per_step = cfg.c * n * groups_per_step
+    value = whole_job_value(world, elems_per_step, args.steps, elapsed_ms)
+    e2e_value = whole_job_value(world, elems_per_step, e2e_steps, e2e_ms)
+    abytes = algorithmic_bytes(n, cfg.c * fuse_t, gbytes)
+    peak, peak_kind = hbm_peak()
+    achieved = abytes / (kern_ms * 1e-3) / 1e9
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": "%s: N=%d fp32 parameters (AlexNet-like layout), lambda=%d, n=%d, c=%d %s gradients "
+                        "per update, T=%d updates per kernel pass" % (cfg.name, n, cfg.num_learners, cfg.n, cfg.c,
+                                                                    cfg.grad_dtype, fuse_t),
+            "num_params": n, "lambda": cfg.num_learners, "n": cfg.n, "c": cfg.c, "fuse_t": fuse_t,
+            "grad_dtype": cfg.grad_dtype, "arrivals": cfg.arrival_model, "alpha0": cfg.alpha0,
+            "momentum": cfg.momentum, "weight_decay": cfg.weight_decay, "modulation": cfg.modulation,
+            "parallelism": "replicas only (independent servers, no data-path collective)" if world > 1 else "1 GPU",
+            "l2": "inputs larger than L2: each step streams %.2f GB from %d rotating gradient buffers"
+                  % (abytes / 1e9, pool_n),
+        },
+        "hbm_gbs": world * abytes * args.steps / (elapsed_ms * 1e-3) / 1e9,
+        "gpu_launches": int(launches),
+        "clocks": clocks.summary(),
+        "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
+                "h2d_bytes_per_step": cfg.c * fuse_t * n * gbytes, "d2h_bytes_per_step": n * 4,
+                "ms_per_step": e2e_ms / e2e_steps},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": TRAFFIC.get(cfg.name), "of": peak_kind,
+                     "kernel_ms": kern_ms, "algorithmic_bytes": abytes},
+    }
+    ps.destroy()
+    return result
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/; None until a capture of the current kernel exists.
+TRAFFIC = {}
+
+
+# ----------------------------------------------------------------------------- oracle arms
+def oracle_sample(cfg, sample_params: int, updates: int, rotate: int = 8):
+    """Time the CPU reference, as it stands, on `updates` updates over the first `sample_params`
+    elements of the workload.  Returns (grad elements per second, seconds)."""
+    from oracle import reference as R
+
+    layout = cfg.layout()
+    idx_n = min(sample_params, layout.num_params)
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+    tdt = torch.bfloat16 if cfg.grad_dtype == "bf16" else torch.float32
+    w0 = G.initial_weights(layout, cfg.seed, cfg.weight_std, device=gen_dev)[:idx_n].cpu()
+    grads = []
+    for i in range(rotate):
+        g = G.gradient(cfg.seed, i, 0, idx_n, cfg.grad_std, dtype=tdt, device=gen_dev).cpu()
+        grads.append(g.view(torch.int16).numpy().view(np.uint16) if tdt == torch.bfloat16 else g.numpy())
+    ref = R.ReferencePS(idx_n, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
+                        R.MOD_INV_STALENESS if cfg.modulation == "inv_staleness" else R.MOD_CONSTANT, 32)
+    ref.set_weights(w0.numpy())
+    steps = step_events(cfg, updates)
+    i = 0
+    t0 = time.perf_counter()
+    for evs in steps:
+        for k, l in evs:
+            if k == arrivals.PULL:
+                ref.pull(l)
+            else:
+                ref.push(l, grads[i % rotate])
+                i += 1
+    dt = time.perf_counter() - t0
+    assert ref.timestamp == updates
+    return cfg.c * idx_n * updates / dt, dt
+
+
+def cpu_baseline(cfg):
+    updates = 24
+    v, dt = oracle_sample(cfg, cfg.layout().num_params, updates)
+    return {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "first %d updates of the workload at full size (%d parameters), fp32 reference, "
+                      "single thread, %.1f s; host has %d cores" % (updates, cfg.layout().num_params, dt, os.cpu_count())}
+
+
+def run_reference(args, cfg):
+    sample_params = 1 << 22
+    v, dt = oracle_sample(cfg, sample_params, args.warmup)       # warm-up steps, untimed in the result
+    v, dt = oracle_sample(cfg, sample_params, args.steps)
+    layout = cfg.layout()
+    sample = ("each step is one update over the first %d of %d parameters, fp32 reference, single thread"
+              % (sample_params, layout.num_params))
+    return {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3 / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "%s (CPU reference on a bounded sample)" % cfg.name, "num_params": layout.num_params,
+                   "lambda": cfg.num_learners, "n": cfg.n, "c": cfg.c, "grad_dtype": cfg.grad_dtype},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large_softsync", choices=sorted(configs.BY_NAME))
+    ap.add_argument("--e2e-steps", type=int, default=12)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    cfg = configs.BY_NAME[args.workload]
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args, cfg)), flush=True)
+        return
+
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    result = run_ours(args, cfg, rank, world, local_rank)
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            result["cpu_baseline"] = cpu_baseline(cfg)
+        print(json.dumps(result), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

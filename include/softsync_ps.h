@@ -1,0 +1,179 @@
+/* softsync_ps.h — C ABI of the n-softsync parameter server (one GPU).
+ *
+ * The calls follow the protocol of "Staleness-aware Async-SGD for Distributed
+ * Deep Learning" (arXiv 1511.05950), Section 2.1: a learner pulls the weights
+ * together with the server's scalar timestamp, computes a gradient, and pushes
+ * it back tagged with that timestamp; the server sums c = floor(lambda / n)
+ * gradients (Section 2.2, Eq. 2), scales each by a learning rate that depends
+ * on its staleness (Section 2.4, Eq. 3) and advances the timestamp by one.
+ *
+ * Conventions
+ *   - Pointers named *_dev are device pointers on the GPU that was current when
+ *     ps_create ran; *_host are host pointers.  The library allocates no device
+ *     memory: weights, momentum and staging slots are bound by the caller.
+ *   - All device work is enqueued on one stream (PS_OPT_STREAM, default: the
+ *     legacy default stream).  Calls return once the work is enqueued unless
+ *     stated otherwise.
+ *   - Every function returns a ps_status; negative values are errors and leave
+ *     the server state unchanged.  Nothing aborts or throws.
+ *   - A handle is not thread-safe: the paper's server handles one blocking call
+ *     at a time (Section 2.3) and so does this one.
+ */
+#ifndef SOFTSYNC_PS_H
+#define SOFTSYNC_PS_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ps_ctx ps_t;               /* opaque; created by ps_create, freed by ps_destroy */
+
+enum ps_modulation {
+    PS_MOD_CONSTANT = 0,                  /* alpha = alpha0 for every gradient (Section 4.3, case (a)) */
+    PS_MOD_INV_STALENESS = 1              /* alpha = alpha0 / max(tau, 1)       (Eq. 3; alpha0 at tau = 0) */
+};
+
+enum ps_status {
+    PS_OK = 0,
+    PS_READY = 1,                         /* ps_push_gradient: this push completed a group of c */
+    PS_ERR_INVALID_ARG = -1,
+    PS_ERR_BAD_LEARNER = -2,              /* learner id outside [0, lambda) */
+    PS_ERR_BAD_TIMESTAMP = -3,            /* ts < 0 or ts > server timestamp: staleness would be negative (Section 2.1) */
+    PS_ERR_NOT_READY = -4,                /* ps_apply_update: no complete group is pending */
+    PS_ERR_QUEUE_FULL = -5,               /* too many unapplied groups, or no free staging slot */
+    PS_ERR_CUDA = -6,                     /* a CUDA call failed; see ps_last_cuda_error */
+    PS_ERR_NOMEM = -7,                    /* host allocation failed */
+    PS_ERR_NO_STATE = -8,                 /* weights/momentum (or staging slots) not bound yet */
+    PS_ERR_LOG_EVICTED = -9               /* requested log range is no longer (or not yet) held */
+};
+
+enum ps_grad_dtype { PS_GRAD_FP32 = 0, PS_GRAD_BF16 = 1 };
+
+enum ps_option {
+    PS_OPT_GRAD_DTYPE = 1,                /* ps_grad_dtype of every pushed gradient; only while nothing is pending */
+    PS_OPT_FUSE_T = 2,                    /* max groups applied by one kernel pass, 1..PS_MAX_FUSE_T (default 1) */
+    PS_OPT_STREAM = 3,                    /* cudaStream_t as an integer (default 0) */
+    PS_OPT_QUEUE_GROUPS = 4,              /* max complete-but-unapplied groups (default 64) */
+    PS_OPT_LOG_UPDATES = 5,               /* how many most recent updates the log keeps (default 65536) */
+    PS_OPT_TIMING = 6,                    /* 1: bracket every update kernel with CUDA events (ps_kernel_time) */
+    PS_OPT_KERNEL = 7,                    /* ps_kernel_choice (default PS_KERNEL_AUTO) */
+    PS_OPT_GRID_BLOCKS = 8,               /* thread blocks per launch; 0 = chosen from the SM count */
+    PS_OPT_BLOCK_THREADS = 9              /* threads per block: 128, 256 or 512; 0 = default */
+};
+
+enum ps_kernel_choice {
+    PS_KERNEL_AUTO = 0,                   /* vector kernel when every pointer is 16-byte aligned, else scalar */
+    PS_KERNEL_SCALAR = 1,                 /* one element per thread and iteration */
+    PS_KERNEL_VECTOR = 2                  /* 16-byte loads and stores */
+};
+
+#define PS_MAX_GROUP 256                  /* largest c = floor(lambda / n) */
+#define PS_MAX_FUSE_T 16                  /* largest temporal-fusion depth */
+#define PS_MAX_ENTRIES 512                /* largest T * c one kernel pass takes; T is clamped to fit */
+
+/* One gradient's part in one weight update; what the server decided, for checking
+ * against Section 2.1 (timestamp, staleness) and Eq. 2-3 (grouping, scale). */
+typedef struct ps_log_entry {
+    int64_t update;                       /* timestamp i the update started from (it produced i + 1) */
+    int64_t push_index;                   /* how many gradients this learner had pushed before */
+    int64_t ts_grad;                      /* j: timestamp of the weights the gradient was computed on */
+    int64_t tau;                          /* staleness i - j >= 0 */
+    int64_t sigma;                        /* staleness used in the learning rate, >= 1 */
+    int32_t learner;
+    int32_t position;                     /* place in the summation order of the group, 0 .. c-1 */
+    float scale;                          /* s = alpha0 / (c * sigma), rounded to fp32 once */
+    float decay;                          /* d = weight_decay * sum of the group's scales (fp32) */
+} ps_log_entry;
+
+/* Section 2.1-2.2.  Creates a server for `num_params` fp32 weights, `lambda` learners and
+ * splitting parameter n (1 <= n <= lambda; c = floor(lambda / n) <= PS_MAX_GROUP).
+ * alpha0: base learning rate; momentum, weight_decay: see ps_apply_update; modulation:
+ * ps_modulation.  Timestamp starts at 0.  The handle is owned by the library. */
+int ps_create(ps_t **out, int64_t num_params, int lambda, int n,
+              float alpha0, float momentum, float weight_decay, int modulation);
+
+/* Frees the handle (not the caller's device buffers).  Waits for enqueued work first. */
+int ps_destroy(ps_t *ps);
+
+/* Binds caller-owned device buffers of num_params fp32 each: weights theta and momentum v.
+ * They must stay valid until ps_destroy.  4-byte alignment is enough; 16-byte alignment
+ * enables the vector kernel.  Does not touch their contents. */
+int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev);
+
+/* Sets theta_0 (copied from w_src, host memory if src_is_host != 0, else device), zeroes the
+ * momentum, resets the timestamp to 0 and drops pending gradients and the log. */
+int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host);
+
+/* Binds `num_slots` caller-owned device slots of `slot_bytes` each (a multiple of 16, at least
+ * num_params * gradient size; base 16-byte aligned) that ps_push_gradient_host copies into. */
+int ps_bind_staging(ps_t *ps, void *slots_dev, int64_t slot_bytes, int num_slots);
+
+int ps_set_option(ps_t *ps, int key, int64_t value);
+int ps_get_option(ps_t *ps, int key, int64_t *value);
+
+/* pullWeights (Section 2.1): *ts receives the server timestamp i a gradient computed on these
+ * weights must carry.  If out_dev != NULL, every complete pending group is applied first and
+ * theta_i (num_params fp32) is copied to out_dev on the stream, so the weights always belong to
+ * the returned timestamp.  out_dev == NULL returns the timestamp only. */
+int ps_pull_weights(ps_t *ps, float *out_dev, int64_t *ts);
+
+/* Same, into host memory; returns after the copy has completed. */
+int ps_pull_weights_host(ps_t *ps, float *out_host, int64_t *ts);
+
+/* pushGradient + the bookkeeping half of sumGradients (Section 2.1, 2.2).  grad_dev: num_params
+ * values of the configured dtype, BORROWED: it must stay valid and unchanged until the
+ * ps_apply_update that consumes it has finished on the stream.  ts: the timestamp the learner
+ * pulled.  Staleness tau = i - ts is taken against the server timestamp i at this call (the
+ * number of complete groups so far).  Returns PS_READY if the gradient completed a group of c,
+ * else PS_OK. */
+int ps_push_gradient(ps_t *ps, int learner, const void *grad_dev, int64_t ts);
+
+/* Same for a gradient in host memory: it is copied (cudaMemcpyAsync on the stream) into a free
+ * staging slot, which is released when the update that consumes it has been enqueued.  The host
+ * buffer may be reused when the call returns only if it is pageable; pinned buffers must stay
+ * unchanged until the stream has passed the copy. */
+int ps_push_gradient_host(ps_t *ps, int learner, const void *grad_host, int64_t ts);
+
+/* applyUpdate fused with sumGradients (Section 2.1; Eq. 2 with the learning rate of Eq. 3):
+ * takes up to PS_OPT_FUSE_T complete groups, oldest first, and applies them in ONE kernel pass
+ * that reads theta and v once, reads every gradient of those groups once, and writes theta and
+ * v once.  Per element and per group, in fp32 with separately rounded multiplies and adds:
+ *     acc = s_1 g_1 + s_2 g_2 + ... + s_c g_c     (ascending learner id, then push index)
+ *     v   = momentum * v + (acc + d * theta)
+ *     theta = theta - v
+ * with s_l = alpha0 / (c * sigma_l) and d = weight_decay * sum_l s_l.  Advances the applied
+ * timestamp by the number of groups and appends to the log.  Returns that number (>= 1) or
+ * PS_ERR_NOT_READY. */
+int ps_apply_update(ps_t *ps);
+
+/* Applies every complete pending group (repeated ps_apply_update).  Returns the number applied (>= 0). */
+int ps_flush(ps_t *ps);
+
+/* Blocks until the stream has finished everything this handle enqueued. */
+int ps_synchronize(ps_t *ps);
+
+/* Copies the log entries of updates [first_update, first_update + count) to out_host
+ * (count * c entries, update-major, in summation order). */
+int ps_get_update_log(ps_t *ps, int64_t first_update, int64_t count, ps_log_entry *out_host);
+
+/* Device pointers of the bound state and both clocks: ts_applied counts updates whose kernel has
+ * been enqueued; ts_logical = ts_applied + complete pending groups (what ps_pull_weights returns).
+ * Any output pointer may be NULL. */
+int ps_peek_state(ps_t *ps, const float **w_dev, const float **v_dev,
+                  int64_t *ts_applied, int64_t *ts_logical);
+
+/* With PS_OPT_TIMING = 1: waits for the stream, then returns the summed CUDA-event duration of the
+ * update kernels launched since the last call and their number.  Either pointer may be NULL. */
+int ps_kernel_time(ps_t *ps, double *total_ms, int64_t *launches);
+
+/* cudaError_t of the most recent failed CUDA call made for this handle (0 if none). */
+int ps_last_cuda_error(ps_t *ps);
+
+const char *ps_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOFTSYNC_PS_H */

@@ -1,0 +1,271 @@
+"""ctypes binding of libsoftsync_ps.so: argument marshalling only.
+
+Every step of the parameter-server path (timestamps, staleness, grouping, the
+scale table, the fused update kernel) runs inside the C-ABI library declared in
+include/softsync_ps.h.  PyTorch is used here for device memory and streams.
+There is no CPU fallback: if the library has not been built, importing this
+module raises.
+"""
+from __future__ import annotations
+
+import collections
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+# ---- constants mirrored from include/softsync_ps.h ---------------------------
+PS_MOD_CONSTANT, PS_MOD_INV_STALENESS = 0, 1
+PS_OK, PS_READY = 0, 1
+PS_ERR_INVALID_ARG, PS_ERR_BAD_LEARNER, PS_ERR_BAD_TIMESTAMP, PS_ERR_NOT_READY = -1, -2, -3, -4
+PS_ERR_QUEUE_FULL, PS_ERR_CUDA, PS_ERR_NOMEM, PS_ERR_NO_STATE, PS_ERR_LOG_EVICTED = -5, -6, -7, -8, -9
+PS_GRAD_FP32, PS_GRAD_BF16 = 0, 1
+(PS_OPT_GRAD_DTYPE, PS_OPT_FUSE_T, PS_OPT_STREAM, PS_OPT_QUEUE_GROUPS, PS_OPT_LOG_UPDATES,
+ PS_OPT_TIMING, PS_OPT_KERNEL, PS_OPT_GRID_BLOCKS, PS_OPT_BLOCK_THREADS) = range(1, 10)
+PS_KERNEL_AUTO, PS_KERNEL_SCALAR, PS_KERNEL_VECTOR = 0, 1, 2
+PS_MAX_GROUP, PS_MAX_FUSE_T, PS_MAX_ENTRIES = 256, 16, 512
+
+MODULATIONS = {"constant": PS_MOD_CONSTANT, "inv_staleness": PS_MOD_INV_STALENESS}
+GRAD_DTYPES = {"fp32": PS_GRAD_FP32, "bf16": PS_GRAD_BF16}
+
+LOG_DTYPE = np.dtype([
+    ("update", "<i8"), ("push_index", "<i8"), ("ts_grad", "<i8"), ("tau", "<i8"), ("sigma", "<i8"),
+    ("learner", "<i4"), ("position", "<i4"), ("scale", "<f4"), ("decay", "<f4"),
+], align=True)
+
+EXPORTS = (
+    "ps_create", "ps_destroy", "ps_bind_state", "ps_init_weights", "ps_bind_staging",
+    "ps_set_option", "ps_get_option", "ps_pull_weights", "ps_pull_weights_host",
+    "ps_push_gradient", "ps_push_gradient_host", "ps_apply_update", "ps_flush", "ps_synchronize",
+    "ps_get_update_log", "ps_peek_state", "ps_kernel_time", "ps_last_cuda_error", "ps_status_string",
+)
+
+
+class SoftsyncError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (%d)" % (where, status_string(status), status))
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        raise RuntimeError(
+            "libsoftsync_ps.so is not built (%s). Run `python -m paper_1511_05950_b200.build`; "
+            "there is no CPU fallback." % path)
+    L = C.CDLL(path)
+    vp, i64, i32, f32 = C.c_void_p, C.c_int64, C.c_int, C.c_float
+    sig = {
+        "ps_create": [C.POINTER(vp), i64, i32, i32, f32, f32, f32, i32],
+        "ps_destroy": [vp],
+        "ps_bind_state": [vp, vp, vp],
+        "ps_init_weights": [vp, vp, i32],
+        "ps_bind_staging": [vp, vp, i64, i32],
+        "ps_set_option": [vp, i32, i64],
+        "ps_get_option": [vp, i32, C.POINTER(i64)],
+        "ps_pull_weights": [vp, vp, C.POINTER(i64)],
+        "ps_pull_weights_host": [vp, vp, C.POINTER(i64)],
+        "ps_push_gradient": [vp, i32, vp, i64],
+        "ps_push_gradient_host": [vp, i32, vp, i64],
+        "ps_apply_update": [vp],
+        "ps_flush": [vp],
+        "ps_synchronize": [vp],
+        "ps_get_update_log": [vp, i64, i64, vp],
+        "ps_peek_state": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), C.POINTER(i64)],
+        "ps_kernel_time": [vp, C.POINTER(C.c_double), C.POINTER(i64)],
+        "ps_last_cuda_error": [vp],
+        "ps_status_string": [i32],
+    }
+    for name, argtypes in sig.items():
+        fn = getattr(L, name)
+        fn.argtypes = argtypes
+        fn.restype = C.c_char_p if name == "ps_status_string" else C.c_int
+    assert LOG_DTYPE.itemsize == 56
+    return L
+
+
+lib = _load()
+
+# The C entry points under their own names, for callers that want the raw ABI.
+ps_create = lib.ps_create
+ps_destroy = lib.ps_destroy
+ps_bind_state = lib.ps_bind_state
+ps_init_weights = lib.ps_init_weights
+ps_bind_staging = lib.ps_bind_staging
+ps_set_option = lib.ps_set_option
+ps_get_option = lib.ps_get_option
+ps_pull_weights = lib.ps_pull_weights
+ps_pull_weights_host = lib.ps_pull_weights_host
+ps_push_gradient = lib.ps_push_gradient
+ps_push_gradient_host = lib.ps_push_gradient_host
+ps_apply_update = lib.ps_apply_update
+ps_flush = lib.ps_flush
+ps_synchronize = lib.ps_synchronize
+ps_get_update_log = lib.ps_get_update_log
+ps_peek_state = lib.ps_peek_state
+ps_kernel_time = lib.ps_kernel_time
+ps_last_cuda_error = lib.ps_last_cuda_error
+
+
+def status_string(status: int) -> str:
+    return lib.ps_status_string(status).decode()
+
+
+def _check(status: int, where: str) -> int:
+    if status < 0:
+        raise SoftsyncError(status, where)
+    return status
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+class ParameterServer:
+    """One n-softsync parameter server on the current CUDA device.
+
+    Owns the device memory (torch tensors) that the library is bound to and
+    keeps pushed gradient tensors alive until the update that consumes them
+    has been enqueued.  Method names follow the C ABI.
+    """
+
+    def __init__(self, num_params: int, num_learners: int, n: int, alpha0: float, momentum: float = 0.0,
+                 weight_decay: float = 0.0, modulation: str = "inv_staleness", grad_dtype: str = "fp32",
+                 fuse_t: int = 1, device: Optional[torch.device] = None,
+                 state: Optional[Tuple[torch.Tensor, torch.Tensor]] = None, allocate: bool = True):
+        self._h = C.c_void_p()
+        self.num_params = int(num_params)
+        self.c = num_learners // n if n >= 1 else 0
+        self.grad_dtype = grad_dtype
+        self._held = collections.deque()
+        self._staging = None
+        self.w = self.v = None
+        if device is None and (allocate or state is not None) and num_params > 0:
+            device = torch.device("cuda", torch.cuda.current_device())
+        self.device = device
+        ctx = torch.cuda.device(device) if device is not None and device.type == "cuda" else _NullCtx()
+        with ctx:
+            _check(ps_create(C.byref(self._h), num_params, num_learners, n, alpha0, momentum, weight_decay,
+                             MODULATIONS[modulation]), "ps_create")
+        if state is not None:
+            self.bind_state(*state)
+        elif allocate and num_params > 0:
+            self.bind_state(torch.empty(num_params, dtype=torch.float32, device=device),
+                            torch.empty(num_params, dtype=torch.float32, device=device))
+        if grad_dtype != "fp32":
+            self.set_option(PS_OPT_GRAD_DTYPE, GRAD_DTYPES[grad_dtype])
+        if fuse_t != 1:
+            self.set_option(PS_OPT_FUSE_T, fuse_t)
+        if device is not None and device.type == "cuda":
+            self.set_option(PS_OPT_STREAM, torch.cuda.current_stream(device).cuda_stream)
+
+    # -- lifetime -------------------------------------------------------------
+    def destroy(self) -> None:
+        if self._h:
+            _check(ps_destroy(self._h), "ps_destroy")
+            self._h = C.c_void_p()
+            self._held.clear()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    # -- set-up ---------------------------------------------------------------
+    def bind_state(self, w: torch.Tensor, v: torch.Tensor) -> None:
+        assert w.dtype == torch.float32 and v.dtype == torch.float32
+        assert w.numel() >= self.num_params and v.numel() >= self.num_params
+        _check(ps_bind_state(self._h, w.data_ptr(), v.data_ptr()), "ps_bind_state")
+        self.w, self.v = w, v
+
+    def init_weights(self, w0: torch.Tensor) -> None:
+        assert w0.dtype == torch.float32 and w0.is_contiguous() and w0.numel() == self.num_params
+        _check(ps_init_weights(self._h, w0.data_ptr(), 0 if w0.is_cuda else 1), "ps_init_weights")
+        self._held.clear()
+
+    def bind_staging(self, num_slots: int) -> None:
+        elem = 2 if self.grad_dtype == "bf16" else 4
+        slot_bytes = (self.num_params * elem + 255) // 256 * 256
+        buf = torch.empty(max(1, slot_bytes * num_slots), dtype=torch.uint8, device=self.device)
+        _check(ps_bind_staging(self._h, buf.data_ptr(), slot_bytes, num_slots), "ps_bind_staging")
+        self._staging = buf
+
+    def set_option(self, key: int, value: int) -> None:
+        _check(ps_set_option(self._h, key, int(value)), "ps_set_option")
+
+    def get_option(self, key: int) -> int:
+        out = C.c_int64()
+        _check(ps_get_option(self._h, key, C.byref(out)), "ps_get_option")
+        return out.value
+
+    # -- the protocol ----------------------------------------------------------
+    def pull_weights(self, out: Optional[torch.Tensor] = None) -> int:
+        """Timestamp a gradient computed from now on must carry; fills `out` with the weights if given."""
+        ts = C.c_int64()
+        if out is not None and not out.is_cuda:
+            assert out.dtype == torch.float32 and out.is_contiguous()
+            _check(ps_pull_weights_host(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host")
+            self._held.clear()
+        else:
+            _check(ps_pull_weights(self._h, _ptr(out), C.byref(ts)), "ps_pull_weights")
+            if out is not None:
+                self._held.clear()
+        return ts.value
+
+    def push_gradient(self, learner: int, grad: torch.Tensor, ts: int) -> bool:
+        """True if this push completed a group of c (an update can be applied)."""
+        if grad.is_cuda:
+            r = _check(ps_push_gradient(self._h, learner, grad.data_ptr(), ts), "ps_push_gradient")
+            self._held.append(grad)
+        else:
+            r = _check(ps_push_gradient_host(self._h, learner, grad.data_ptr(), ts), "ps_push_gradient_host")
+            self._held.append(None)
+        return r == PS_READY
+
+    def apply_update(self) -> int:
+        done = _check(ps_apply_update(self._h), "ps_apply_update")
+        for _ in range(done * self.c):
+            self._held.popleft()
+        return done
+
+    def flush(self) -> int:
+        done = _check(ps_flush(self._h), "ps_flush")
+        for _ in range(done * self.c):
+            self._held.popleft()
+        return done
+
+    def synchronize(self) -> None:
+        _check(ps_synchronize(self._h), "ps_synchronize")
+
+    # -- inspection -------------------------------------------------------------
+    def timestamps(self) -> Tuple[int, int]:
+        """(applied, logical)."""
+        a, l = C.c_int64(), C.c_int64()
+        _check(ps_peek_state(self._h, None, None, C.byref(a), C.byref(l)), "ps_peek_state")
+        return a.value, l.value
+
+    def update_log(self, first_update: int = 0, count: Optional[int] = None) -> np.ndarray:
+        if count is None:
+            count = self.timestamps()[0] - first_update
+        out = np.empty(count * self.c, dtype=LOG_DTYPE)
+        _check(ps_get_update_log(self._h, first_update, count, out.ctypes.data if out.size else None),
+               "ps_get_update_log")
+        return out
+
+    def kernel_time(self) -> Tuple[float, int]:
+        ms, n = C.c_double(), C.c_int64()
+        _check(ps_kernel_time(self._h, C.byref(ms), C.byref(n)), "ps_kernel_time")
+        return ms.value, n.value
+
+
+class _NullCtx:
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        return False

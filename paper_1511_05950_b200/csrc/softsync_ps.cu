@@ -1,0 +1,539 @@
+// C ABI and host-side protocol state of the n-softsync parameter server
+// (arXiv 1511.05950, Section 2.1-2.4).  The O(N) work is in update_kernels.cuh;
+// this file keeps the scalar timestamp clock, computes staleness at push time,
+// groups gradients first come first grouped, builds the per-launch scale table
+// and records what it decided in the update log.
+#include "../../include/softsync_ps.h"
+#include "update_kernels.cuh"
+
+#include <algorithm>
+#include <deque>
+#include <mutex>
+#include <new>
+#include <unordered_set>
+#include <vector>
+
+namespace {
+
+using softsync::GradBf16;
+using softsync::GradFp32;
+using softsync::LaunchParams;
+
+struct Entry {                 // one pushed gradient waiting for its update
+    int32_t learner;
+    int64_t push_index, ts_grad, tau, sigma;
+    const void *grad;
+    int slot;                  // staging slot it occupies, -1 if borrowed from the caller
+};
+
+struct TimedLaunch { cudaEvent_t start, stop; };
+constexpr size_t kMaxTimedLaunches = 1 << 16;   // launches held between two ps_kernel_time calls
+
+}  // namespace
+
+struct ps_ctx {
+    int64_t n = 0;
+    int lambda = 0, split = 0, c = 0, modulation = 0;
+    float alpha0 = 0, momentum = 0, weight_decay = 0;
+    int device = 0;
+
+    float *w = nullptr, *v = nullptr;
+    char *staging = nullptr;
+    int64_t slot_bytes = 0;
+    std::vector<int> free_slots;
+    int num_slots = 0;
+
+    int grad_dtype = PS_GRAD_FP32;
+    int fuse_t = 1;
+    cudaStream_t stream = nullptr;
+    int64_t queue_groups = 64;
+    int64_t log_updates = 65536;
+    int timing = 0, kernel_choice = PS_KERNEL_AUTO, grid_blocks = 0, block_threads = 0;
+    int sm_count = 0;
+
+    int64_t ts_applied = 0;                // updates whose kernel has been enqueued
+    std::deque<std::vector<Entry>> ready;  // complete groups, oldest first
+    std::vector<Entry> filling;            // the group being collected (< c entries)
+    std::vector<int64_t> push_count;       // per learner
+
+    std::deque<ps_log_entry> log;          // c entries per update, oldest first
+    int64_t log_first_update = 0;
+
+    std::vector<TimedLaunch> timed, spare_events;
+    int last_cuda_error = 0;
+};
+
+namespace {
+
+std::mutex g_live_mutex;
+std::unordered_set<ps_ctx *> g_live;       // handles that ps_create returned and ps_destroy has not seen
+
+bool is_live(ps_ctx *ps)
+{
+    if (!ps) return false;
+    std::lock_guard<std::mutex> lock(g_live_mutex);
+    return g_live.count(ps) != 0;
+}
+
+int cuda_fail(ps_ctx *ps, cudaError_t e)
+{
+    ps->last_cuda_error = static_cast<int>(e);
+    return PS_ERR_CUDA;
+}
+#define PS_CUDA(ps, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail((ps), e_); } while (0)
+
+size_t grad_elem_bytes(const ps_ctx *ps) { return ps->grad_dtype == PS_GRAD_BF16 ? 2 : 4; }
+
+int64_t ts_logical(const ps_ctx *ps) { return ps->ts_applied + static_cast<int64_t>(ps->ready.size()); }
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Summation order inside a group: ascending learner id, then push index.
+bool entry_before(const Entry &a, const Entry &b)
+{
+    return a.learner != b.learner ? a.learner < b.learner : a.push_index < b.push_index;
+}
+
+template <typename GT, int VEC, int K, int MAXE>
+cudaError_t launch_variant(const LaunchParams<MAXE> &p, int blocks, int threads, cudaStream_t stream)
+{
+    softsync::softsync_update_kernel<GT, VEC, K, MAXE><<<blocks, threads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+template <int MAXE>
+cudaError_t launch_update(ps_ctx *ps, const LaunchParams<MAXE> &p, bool vector_ok)
+{
+    const bool bf16 = ps->grad_dtype == PS_GRAD_BF16;
+    const int vec = vector_ok ? (bf16 ? 8 : 4) : 1;
+    const int threads = ps->block_threads ? ps->block_threads : 256;
+    const long long frags = std::max<long long>(1, (p.n + vec - 1) / vec);
+    long long blocks = (frags + threads - 1) / threads;
+    const long long cap = ps->grid_blocks ? ps->grid_blocks
+                                          : static_cast<long long>(ps->sm_count) * (2048 / threads) * 4;
+    blocks = std::max<long long>(1, std::min(blocks, cap));
+    const int b = static_cast<int>(blocks);
+    if (vector_ok)
+        return bf16 ? launch_variant<GradBf16, 8, 8, MAXE>(p, b, threads, ps->stream)
+                    : launch_variant<GradFp32, 4, 8, MAXE>(p, b, threads, ps->stream);
+    return bf16 ? launch_variant<GradBf16, 1, 8, MAXE>(p, b, threads, ps->stream)
+                : launch_variant<GradFp32, 1, 8, MAXE>(p, b, threads, ps->stream);
+}
+
+// Fills the scale table of one launch (Eq. 3 folded with the 1/c of Eq. 2) for the `T`
+// oldest complete groups and the log entries that describe them.
+template <int MAXE>
+void build_launch(ps_ctx *ps, int T, LaunchParams<MAXE> &p, std::vector<ps_log_entry> &entries, bool &vector_ok)
+{
+    p.w = ps->w; p.v = ps->v; p.n = ps->n;
+    p.momentum = ps->momentum; p.T = T; p.c = ps->c;
+    vector_ok = aligned16(ps->w) && aligned16(ps->v);
+    const double alpha0 = static_cast<double>(ps->alpha0);
+    const double wd = static_cast<double>(ps->weight_decay);
+    for (int t = 0; t < T; ++t) {
+        std::vector<Entry> &grp = ps->ready[t];
+        std::stable_sort(grp.begin(), grp.end(), entry_before);
+        double sum = 0.0;
+        for (int l = 0; l < ps->c; ++l) {
+            const Entry &en = grp[l];
+            const float s = static_cast<float>(alpha0 / (static_cast<double>(ps->c) * static_cast<double>(en.sigma)));
+            p.s[t * ps->c + l] = s;
+            p.g[t * ps->c + l] = en.grad;
+            vector_ok = vector_ok && aligned16(en.grad);
+            sum += static_cast<double>(s);
+        }
+        const float d = static_cast<float>(wd * sum);   // every gradient carries + wd * theta
+        p.d[t] = d;
+        for (int l = 0; l < ps->c; ++l) {
+            const Entry &en = grp[l];
+            ps_log_entry le;
+            le.update = ps->ts_applied + t;
+            le.push_index = en.push_index; le.ts_grad = en.ts_grad; le.tau = en.tau; le.sigma = en.sigma;
+            le.learner = en.learner; le.position = l;
+            le.scale = p.s[t * ps->c + l]; le.decay = d;
+            entries.push_back(le);
+        }
+    }
+}
+
+int take_events(ps_ctx *ps, TimedLaunch &tl)
+{
+    if (!ps->spare_events.empty()) { tl = ps->spare_events.back(); ps->spare_events.pop_back(); return PS_OK; }
+    PS_CUDA(ps, cudaEventCreate(&tl.start));
+    PS_CUDA(ps, cudaEventCreate(&tl.stop));
+    return PS_OK;
+}
+
+template <int MAXE>
+int apply_groups(ps_ctx *ps, int T)
+{
+    LaunchParams<MAXE> p;
+    std::vector<ps_log_entry> entries;
+    entries.reserve(static_cast<size_t>(T) * ps->c);
+    bool vector_ok = false;
+    build_launch<MAXE>(ps, T, p, entries, vector_ok);
+    if (ps->kernel_choice == PS_KERNEL_SCALAR) vector_ok = false;
+    if (ps->kernel_choice == PS_KERNEL_VECTOR && !vector_ok) return PS_ERR_INVALID_ARG;
+
+    if (ps->n > 0) {
+        TimedLaunch tl{};
+        const bool timed = ps->timing && ps->timed.size() < kMaxTimedLaunches;
+        if (timed) {
+            int rc = take_events(ps, tl);
+            if (rc != PS_OK) return rc;
+            PS_CUDA(ps, cudaEventRecord(tl.start, ps->stream));
+        }
+        PS_CUDA(ps, launch_update<MAXE>(ps, p, vector_ok));
+        if (timed) {
+            PS_CUDA(ps, cudaEventRecord(tl.stop, ps->stream));
+            ps->timed.push_back(tl);
+        }
+    }
+    // the launch is enqueued: advance the clock, release slots, publish the log
+    for (int t = 0; t < T; ++t) {
+        for (const Entry &en : ps->ready.front())
+            if (en.slot >= 0) ps->free_slots.push_back(en.slot);
+        ps->ready.pop_front();
+    }
+    ps->ts_applied += T;
+    for (const ps_log_entry &le : entries) ps->log.push_back(le);
+    const int64_t held = static_cast<int64_t>(ps->log.size()) / ps->c;
+    if (held > ps->log_updates) {
+        const int64_t drop = held - ps->log_updates;
+        ps->log.erase(ps->log.begin(), ps->log.begin() + drop * ps->c);
+        ps->log_first_update += drop;
+    }
+    return T;
+}
+
+int apply_some(ps_ctx *ps)
+{
+    if (ps->n > 0 && (!ps->w || !ps->v)) return PS_ERR_NO_STATE;
+    if (ps->ready.empty()) return PS_ERR_NOT_READY;
+    int T = static_cast<int>(std::min<int64_t>(ps->fuse_t, static_cast<int64_t>(ps->ready.size())));
+    T = std::min(T, std::max(1, PS_MAX_ENTRIES / ps->c));
+    return T * ps->c <= 16 ? apply_groups<16>(ps, T) : apply_groups<PS_MAX_ENTRIES>(ps, T);
+}
+
+int push_common(ps_ctx *ps, int learner, const void *grad_dev, int64_t ts, int slot)
+{
+    const int64_t i = ts_logical(ps);
+    Entry en;
+    en.learner = learner;
+    en.push_index = ps->push_count[learner];
+    en.ts_grad = ts;
+    en.tau = i - ts;                                      // staleness (Section 2.1)
+    en.sigma = ps->modulation == PS_MOD_INV_STALENESS ? std::max<int64_t>(en.tau, 1) : 1;
+    en.grad = grad_dev;
+    en.slot = slot;
+    ps->push_count[learner] += 1;
+    ps->filling.push_back(en);
+    if (static_cast<int>(ps->filling.size()) == ps->c) {  // group of c complete: the clock moves on
+        ps->ready.push_back(std::move(ps->filling));
+        ps->filling.clear();
+        ps->filling.reserve(ps->c);
+        return PS_READY;
+    }
+    return PS_OK;
+}
+
+int check_push(ps_ctx *ps, int learner, const void *grad, int64_t ts)
+{
+    if (!grad) return PS_ERR_INVALID_ARG;
+    if (learner < 0 || learner >= ps->lambda) return PS_ERR_BAD_LEARNER;
+    if (ts < 0 || ts > ts_logical(ps)) return PS_ERR_BAD_TIMESTAMP;
+    if (static_cast<int64_t>(ps->ready.size()) >= ps->queue_groups) return PS_ERR_QUEUE_FULL;
+    return PS_OK;
+}
+
+void release_events(ps_ctx *ps)
+{
+    for (auto &tl : ps->timed) ps->spare_events.push_back(tl);
+    ps->timed.clear();
+}
+
+}  // namespace
+
+extern "C" {
+
+int ps_create(ps_t **out, int64_t num_params, int lambda, int n,
+              float alpha0, float momentum, float weight_decay, int modulation)
+{
+    if (!out) return PS_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (num_params < 0 || lambda < 1 || n < 1 || n > lambda) return PS_ERR_INVALID_ARG;
+    if (modulation != PS_MOD_CONSTANT && modulation != PS_MOD_INV_STALENESS) return PS_ERR_INVALID_ARG;
+    if (lambda / n > PS_MAX_GROUP) return PS_ERR_INVALID_ARG;
+    if (!(alpha0 == alpha0) || !(momentum == momentum) || !(weight_decay == weight_decay)) return PS_ERR_INVALID_ARG;
+    ps_ctx *ps = new (std::nothrow) ps_ctx;
+    if (!ps) return PS_ERR_NOMEM;
+    ps->n = num_params; ps->lambda = lambda; ps->split = n; ps->c = lambda / n;   // Eq. 2: c = floor(lambda / n)
+    ps->alpha0 = alpha0; ps->momentum = momentum; ps->weight_decay = weight_decay;
+    ps->modulation = modulation;
+    cudaError_t e = cudaGetDevice(&ps->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ps->sm_count, cudaDevAttrMultiProcessorCount, ps->device);
+    if (e != cudaSuccess) {
+        // No usable GPU and there is no CPU path: only a server with zero parameters
+        // (protocol bookkeeping alone, nothing to launch) may exist without one.
+        cudaGetLastError();
+        if (num_params > 0) { delete ps; return PS_ERR_CUDA; }
+        ps->device = -1; ps->sm_count = 1;
+    }
+    try {
+        ps->push_count.assign(lambda, 0);
+        ps->filling.reserve(ps->c);
+    } catch (const std::bad_alloc &) { delete ps; return PS_ERR_NOMEM; }
+    {
+        std::lock_guard<std::mutex> lock(g_live_mutex);
+        g_live.insert(ps);
+    }
+    *out = ps;
+    return PS_OK;
+}
+
+int ps_destroy(ps_t *ps)
+{
+    {
+        std::lock_guard<std::mutex> lock(g_live_mutex);
+        if (!ps || !g_live.erase(ps)) return PS_ERR_INVALID_ARG;
+    }
+    if (ps->device >= 0) cudaStreamSynchronize(ps->stream);
+    release_events(ps);
+    for (auto &tl : ps->spare_events) { cudaEventDestroy(tl.start); cudaEventDestroy(tl.stop); }
+    delete ps;
+    return PS_OK;
+}
+
+int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev)
+{
+    if (!is_live(ps) || !w_dev || !v_dev || w_dev == v_dev) return PS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(w_dev) & 3u) || (reinterpret_cast<uintptr_t>(v_dev) & 3u)) return PS_ERR_INVALID_ARG;
+    if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+    ps->w = w_dev; ps->v = v_dev;
+    return PS_OK;
+}
+
+int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host)
+{
+    if (!is_live(ps) || !w_src) return PS_ERR_INVALID_ARG;
+    if (!ps->w || !ps->v) return PS_ERR_NO_STATE;
+    const size_t bytes = static_cast<size_t>(ps->n) * sizeof(float);
+    if (bytes) {
+        PS_CUDA(ps, cudaMemcpyAsync(ps->w, w_src, bytes, src_is_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, ps->stream));
+        PS_CUDA(ps, cudaMemsetAsync(ps->v, 0, bytes, ps->stream));
+        if (src_is_host) PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+    }
+    for (auto &grp : ps->ready) for (const Entry &en : grp) if (en.slot >= 0) ps->free_slots.push_back(en.slot);
+    for (const Entry &en : ps->filling) if (en.slot >= 0) ps->free_slots.push_back(en.slot);
+    ps->ready.clear(); ps->filling.clear();
+    std::fill(ps->push_count.begin(), ps->push_count.end(), 0);
+    ps->ts_applied = 0;
+    ps->log.clear(); ps->log_first_update = 0;
+    return PS_OK;
+}
+
+int ps_bind_staging(ps_t *ps, void *slots_dev, int64_t slot_bytes, int num_slots)
+{
+    if (!is_live(ps) || !slots_dev || num_slots < 1 || slot_bytes < 0) return PS_ERR_INVALID_ARG;
+    if (!aligned16(slots_dev) || (slot_bytes & 15)) return PS_ERR_INVALID_ARG;
+    if (slot_bytes < ps->n * static_cast<int64_t>(grad_elem_bytes(ps))) return PS_ERR_INVALID_ARG;
+    if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+    ps->staging = static_cast<char *>(slots_dev);
+    ps->slot_bytes = slot_bytes; ps->num_slots = num_slots;
+    ps->free_slots.clear();
+    for (int s = num_slots - 1; s >= 0; --s) ps->free_slots.push_back(s);
+    return PS_OK;
+}
+
+int ps_set_option(ps_t *ps, int key, int64_t value)
+{
+    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    switch (key) {
+    case PS_OPT_GRAD_DTYPE:
+        if (value != PS_GRAD_FP32 && value != PS_GRAD_BF16) return PS_ERR_INVALID_ARG;
+        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+        if (ps->staging && ps->slot_bytes < ps->n * (value == PS_GRAD_BF16 ? 2 : 4)) return PS_ERR_INVALID_ARG;
+        ps->grad_dtype = static_cast<int>(value); return PS_OK;
+    case PS_OPT_FUSE_T:
+        if (value < 1 || value > PS_MAX_FUSE_T) return PS_ERR_INVALID_ARG;
+        ps->fuse_t = static_cast<int>(value); return PS_OK;
+    case PS_OPT_STREAM:
+        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+        ps->stream = reinterpret_cast<cudaStream_t>(static_cast<uintptr_t>(value)); return PS_OK;
+    case PS_OPT_QUEUE_GROUPS:
+        if (value < 1) return PS_ERR_INVALID_ARG;
+        ps->queue_groups = value; return PS_OK;
+    case PS_OPT_LOG_UPDATES:
+        if (value < 0) return PS_ERR_INVALID_ARG;
+        ps->log_updates = value; return PS_OK;
+    case PS_OPT_TIMING:
+        if (value != 0 && value != 1) return PS_ERR_INVALID_ARG;
+        ps->timing = static_cast<int>(value); return PS_OK;
+    case PS_OPT_KERNEL:
+        if (value < PS_KERNEL_AUTO || value > PS_KERNEL_VECTOR) return PS_ERR_INVALID_ARG;
+        ps->kernel_choice = static_cast<int>(value); return PS_OK;
+    case PS_OPT_GRID_BLOCKS:
+        if (value < 0 || value > 0x7fffffff) return PS_ERR_INVALID_ARG;
+        ps->grid_blocks = static_cast<int>(value); return PS_OK;
+    case PS_OPT_BLOCK_THREADS:
+        if (value != 0 && value != 128 && value != 256 && value != 512) return PS_ERR_INVALID_ARG;
+        ps->block_threads = static_cast<int>(value); return PS_OK;
+    default:
+        return PS_ERR_INVALID_ARG;
+    }
+}
+
+int ps_get_option(ps_t *ps, int key, int64_t *value)
+{
+    if (!is_live(ps) || !value) return PS_ERR_INVALID_ARG;
+    switch (key) {
+    case PS_OPT_GRAD_DTYPE: *value = ps->grad_dtype; return PS_OK;
+    case PS_OPT_FUSE_T: *value = ps->fuse_t; return PS_OK;
+    case PS_OPT_STREAM: *value = static_cast<int64_t>(reinterpret_cast<uintptr_t>(ps->stream)); return PS_OK;
+    case PS_OPT_QUEUE_GROUPS: *value = ps->queue_groups; return PS_OK;
+    case PS_OPT_LOG_UPDATES: *value = ps->log_updates; return PS_OK;
+    case PS_OPT_TIMING: *value = ps->timing; return PS_OK;
+    case PS_OPT_KERNEL: *value = ps->kernel_choice; return PS_OK;
+    case PS_OPT_GRID_BLOCKS: *value = ps->grid_blocks; return PS_OK;
+    case PS_OPT_BLOCK_THREADS: *value = ps->block_threads; return PS_OK;
+    default: return PS_ERR_INVALID_ARG;
+    }
+}
+
+int ps_apply_update(ps_t *ps)
+{
+    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    return apply_some(ps);
+}
+
+int ps_flush(ps_t *ps)
+{
+    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    int total = 0;
+    while (!ps->ready.empty()) {
+        const int r = apply_some(ps);
+        if (r < 0) return r;
+        total += r;
+    }
+    return total;
+}
+
+int ps_pull_weights(ps_t *ps, float *out_dev, int64_t *ts)
+{
+    if (!is_live(ps) || !ts) return PS_ERR_INVALID_ARG;
+    if (out_dev) {
+        if (ps->n > 0 && (!ps->w || !ps->v)) return PS_ERR_NO_STATE;
+        const int r = ps_flush(ps);                       // weights must belong to the returned timestamp
+        if (r < 0) return r;
+        if (ps->n) PS_CUDA(ps, cudaMemcpyAsync(out_dev, ps->w, static_cast<size_t>(ps->n) * sizeof(float),
+                                               cudaMemcpyDeviceToDevice, ps->stream));
+    }
+    *ts = ts_logical(ps);
+    return PS_OK;
+}
+
+int ps_pull_weights_host(ps_t *ps, float *out_host, int64_t *ts)
+{
+    if (!is_live(ps) || !ts || !out_host) return PS_ERR_INVALID_ARG;
+    if (!ps->w || !ps->v) return PS_ERR_NO_STATE;
+    const int r = ps_flush(ps);
+    if (r < 0) return r;
+    if (ps->n) PS_CUDA(ps, cudaMemcpyAsync(out_host, ps->w, static_cast<size_t>(ps->n) * sizeof(float),
+                                           cudaMemcpyDeviceToHost, ps->stream));
+    PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+    *ts = ts_logical(ps);
+    return PS_OK;
+}
+
+int ps_push_gradient(ps_t *ps, int learner, const void *grad_dev, int64_t ts)
+{
+    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    const int rc = check_push(ps, learner, grad_dev, ts);
+    if (rc != PS_OK) return rc;
+    if (reinterpret_cast<uintptr_t>(grad_dev) & (grad_elem_bytes(ps) - 1)) return PS_ERR_INVALID_ARG;
+    return push_common(ps, learner, grad_dev, ts, -1);
+}
+
+int ps_push_gradient_host(ps_t *ps, int learner, const void *grad_host, int64_t ts)
+{
+    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    const int rc = check_push(ps, learner, grad_host, ts);
+    if (rc != PS_OK) return rc;
+    if (!ps->staging) return PS_ERR_NO_STATE;
+    if (ps->free_slots.empty()) return PS_ERR_QUEUE_FULL;
+    const int slot = ps->free_slots.back();
+    char *dst = ps->staging + static_cast<int64_t>(slot) * ps->slot_bytes;
+    const size_t bytes = static_cast<size_t>(ps->n) * grad_elem_bytes(ps);
+    if (bytes) PS_CUDA(ps, cudaMemcpyAsync(dst, grad_host, bytes, cudaMemcpyHostToDevice, ps->stream));
+    ps->free_slots.pop_back();
+    return push_common(ps, learner, dst, ts, slot);
+}
+
+int ps_synchronize(ps_t *ps)
+{
+    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+    return PS_OK;
+}
+
+int ps_get_update_log(ps_t *ps, int64_t first_update, int64_t count, ps_log_entry *out_host)
+{
+    if (!is_live(ps) || count < 0 || (count > 0 && !out_host)) return PS_ERR_INVALID_ARG;
+    const int64_t held = static_cast<int64_t>(ps->log.size()) / ps->c;
+    if (first_update < ps->log_first_update || first_update + count > ps->log_first_update + held)
+        return PS_ERR_LOG_EVICTED;
+    const int64_t off = (first_update - ps->log_first_update) * ps->c;
+    std::copy(ps->log.begin() + off, ps->log.begin() + off + count * ps->c, out_host);
+    return PS_OK;
+}
+
+int ps_peek_state(ps_t *ps, const float **w_dev, const float **v_dev, int64_t *ts_applied, int64_t *ts_log)
+{
+    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    if (w_dev) *w_dev = ps->w;
+    if (v_dev) *v_dev = ps->v;
+    if (ts_applied) *ts_applied = ps->ts_applied;
+    if (ts_log) *ts_log = ts_logical(ps);
+    return PS_OK;
+}
+
+int ps_kernel_time(ps_t *ps, double *total_ms, int64_t *launches)
+{
+    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+    double sum = 0.0;
+    for (const auto &tl : ps->timed) {
+        float ms = 0.f;
+        PS_CUDA(ps, cudaEventElapsedTime(&ms, tl.start, tl.stop));
+        sum += ms;
+    }
+    if (total_ms) *total_ms = sum;
+    if (launches) *launches = static_cast<int64_t>(ps->timed.size());
+    release_events(ps);
+    return PS_OK;
+}
+
+int ps_last_cuda_error(ps_t *ps)
+{
+    return is_live(ps) ? ps->last_cuda_error : 0;
+}
+
+const char *ps_status_string(int status)
+{
+    switch (status) {
+    case PS_OK: return "ok";
+    case PS_READY: return "ready: a group of c gradients is complete";
+    case PS_ERR_INVALID_ARG: return "invalid argument";
+    case PS_ERR_BAD_LEARNER: return "learner id out of range";
+    case PS_ERR_BAD_TIMESTAMP: return "gradient timestamp negative or ahead of the server";
+    case PS_ERR_NOT_READY: return "no complete group is pending";
+    case PS_ERR_QUEUE_FULL: return "too many unapplied groups or no free staging slot";
+    case PS_ERR_CUDA: return "CUDA call failed";
+    case PS_ERR_NOMEM: return "host allocation failed";
+    case PS_ERR_NO_STATE: return "weights, momentum or staging slots not bound";
+    case PS_ERR_LOG_EVICTED: return "log range not held";
+    default: return status > 1 ? "updates applied" : "unknown status";
+    }
+}
+
+}  // extern "C"

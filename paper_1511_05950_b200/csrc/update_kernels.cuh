@@ -1,0 +1,178 @@
+// Fused sumGradients + applyUpdate kernels of the n-softsync parameter server
+// (arXiv 1511.05950, Section 2.1; Eq. 2 with the per-gradient rate of Eq. 3).
+//
+// One pass over the parameter vector: every thread owns VEC consecutive
+// elements, loads theta and v once, streams the T*c gradient values of those
+// elements through registers, applies the T updates in order and stores theta
+// and v once.  The path is HBM-bound (about 0.3 flop per byte), so the work is
+// plain fp32 ALU code around wide coalesced loads; tensor cores have no part.
+//
+// Arithmetic contract (bit-exact, any launch shape): per element and per group
+//     acc = s_1*g_1;  acc = acc + s_l*g_l  (l = 2..c);
+//     t = acc + d*theta;  v = m*v + t;  theta = theta - v
+// with every multiply and add rounded separately (__fmul_rn / __fadd_rn are
+// never contracted into an FMA).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace softsync {
+
+constexpr int kMaxFuseT = 16;
+
+// Everything one launch needs, passed by value in kernel-parameter space: the
+// per-gradient scales s (Eq. 3 folded with the 1/c of Eq. 2), the per-group
+// decay coefficients d and the borrowed gradient pointers, group-major.
+template <int MAXE>
+struct LaunchParams {
+    float *w;
+    float *v;
+    long long n;          // elements
+    float momentum;
+    int T;                // groups in this pass
+    int c;                // gradients per group
+    float d[kMaxFuseT];
+    float s[MAXE];
+    const void *g[MAXE];
+};
+
+struct GradFp32 {};
+struct GradBf16 {};
+
+// ---- raw 16-byte (or scalar) gradient fragments ---------------------------
+template <typename GT, int VEC> struct Raw;
+template <> struct Raw<GradFp32, 4> { float4 q; };
+template <> struct Raw<GradBf16, 8> { uint4 q; };
+template <> struct Raw<GradFp32, 1> { float q; };
+template <> struct Raw<GradBf16, 1> { unsigned short q; };
+
+__device__ __forceinline__ float4 ld_stream_f4(const float4 *p)
+{
+    float4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ uint4 ld_stream_u4(const uint4 *p)
+{
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ void load_raw(Raw<GradFp32, 4> &r, const void *base, long long i)
+{ r.q = ld_stream_f4(reinterpret_cast<const float4 *>(base) + i); }
+__device__ __forceinline__ void load_raw(Raw<GradBf16, 8> &r, const void *base, long long i)
+{ r.q = ld_stream_u4(reinterpret_cast<const uint4 *>(base) + i); }
+__device__ __forceinline__ void load_raw(Raw<GradFp32, 1> &r, const void *base, long long i)
+{ r.q = __ldg(reinterpret_cast<const float *>(base) + i); }
+__device__ __forceinline__ void load_raw(Raw<GradBf16, 1> &r, const void *base, long long i)
+{ r.q = __ldg(reinterpret_cast<const unsigned short *>(base) + i); }
+
+// bf16 is the upper half of an fp32: widening is a shift, exact.
+__device__ __forceinline__ void widen(const Raw<GradFp32, 4> &r, float (&g)[4])
+{ g[0] = r.q.x; g[1] = r.q.y; g[2] = r.q.z; g[3] = r.q.w; }
+__device__ __forceinline__ void widen(const Raw<GradBf16, 8> &r, float (&g)[8])
+{
+    const unsigned u[4] = {r.q.x, r.q.y, r.q.z, r.q.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        g[2 * j] = __uint_as_float(u[j] << 16);
+        g[2 * j + 1] = __uint_as_float(u[j] & 0xFFFF0000u);
+    }
+}
+__device__ __forceinline__ void widen(const Raw<GradFp32, 1> &r, float (&g)[1]) { g[0] = r.q; }
+__device__ __forceinline__ void widen(const Raw<GradBf16, 1> &r, float (&g)[1])
+{ g[0] = __uint_as_float(static_cast<unsigned>(r.q) << 16); }
+
+// ---- theta / v fragments ---------------------------------------------------
+template <int VEC>
+__device__ __forceinline__ void load_state(const float *p, float (&x)[VEC])
+{
+    if constexpr (VEC == 1) {
+        x[0] = *p;
+    } else {
+#pragma unroll
+        for (int j = 0; j < VEC / 4; ++j) {
+            const float4 q = __ldcs(reinterpret_cast<const float4 *>(p) + j);
+            x[4 * j] = q.x; x[4 * j + 1] = q.y; x[4 * j + 2] = q.z; x[4 * j + 3] = q.w;
+        }
+    }
+}
+template <int VEC>
+__device__ __forceinline__ void store_state(float *p, const float (&x)[VEC])
+{
+    if constexpr (VEC == 1) {
+        *p = x[0];
+    } else {
+#pragma unroll
+        for (int j = 0; j < VEC / 4; ++j)
+            __stcs(reinterpret_cast<float4 *>(p) + j, make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]));
+    }
+}
+
+// ---- VEC elements starting at element index first = i * VEC ----------------
+template <typename GT, int VEC, int K, int MAXE>
+__device__ __forceinline__ void update_fragment(const LaunchParams<MAXE> &p, long long i, long long first)
+{
+    float w[VEC], v[VEC], acc[VEC];
+    load_state<VEC>(p.w + first, w);
+    load_state<VEC>(p.v + first, v);
+    const int E = p.T * p.c;
+    const float m = p.momentum;
+    int l = 0, t = 0;
+    for (int e0 = 0; e0 < E; e0 += K) {
+        Raw<GT, VEC> raw[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k)                      // K independent loads in flight
+            if (e0 + k < E) load_raw(raw[k], p.g[e0 + k], i);
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            if (e0 + k < E) {
+                float g[VEC];
+                widen(raw[k], g);
+                const float s = p.s[e0 + k];
+                if (l == 0) {
+#pragma unroll
+                    for (int j = 0; j < VEC; ++j) acc[j] = __fmul_rn(s, g[j]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < VEC; ++j) acc[j] = __fadd_rn(acc[j], __fmul_rn(s, g[j]));
+                }
+                if (++l == p.c) {                        // group complete: one weight update
+                    const float d = p.d[t++];
+                    l = 0;
+#pragma unroll
+                    for (int j = 0; j < VEC; ++j) {
+                        const float tt = __fadd_rn(acc[j], __fmul_rn(d, w[j]));
+                        v[j] = __fadd_rn(__fmul_rn(m, v[j]), tt);
+                        w[j] = __fsub_rn(w[j], v[j]);
+                    }
+                }
+            }
+        }
+    }
+    store_state<VEC>(p.w + first, w);
+    store_state<VEC>(p.v + first, v);
+}
+
+// Grid-stride over fragments of VEC elements; the (n mod VEC) trailing
+// elements are done one by one by the first threads of the grid.
+template <typename GT, int VEC, int K, int MAXE>
+__global__ void softsync_update_kernel(const __grid_constant__ LaunchParams<MAXE> p)
+{
+    const long long nfrag = p.n / VEC;
+    const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = tid; i < nfrag; i += stride)
+        update_fragment<GT, VEC, K, MAXE>(p, i, i * VEC);
+    if constexpr (VEC > 1) {
+        const long long done = nfrag * VEC;
+        if (tid < p.n - done)
+            update_fragment<GT, 1, K, MAXE>(p, done + tid, done + tid);
+    }
+}
+
+}  // namespace softsync

@@ -1,0 +1,126 @@
+"""Drive the CUDA library and the reference with the same seeded inputs (GPU tests only)."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import paper_1511_05950_b200 as P
+from oracle import reference as R
+from tests.helpers import PULL, rel_l2
+from workloads import generators as G
+
+TORCH_DTYPE = {"fp32": torch.float32, "bf16": torch.bfloat16}
+
+
+def as_reference_grad(g: torch.Tensor) -> np.ndarray:
+    """Device gradient -> what the reference's push takes (fp32 values or bf16 bit patterns)."""
+    g = g.detach().cpu()
+    if g.dtype == torch.bfloat16:
+        return g.view(torch.int16).numpy().view(np.uint16)
+    return g.numpy()
+
+
+def replay_gpu(ps: P.ParameterServer, kinds, learners, grad_fn, lazy: bool = False, fuse_t: int = 1):
+    """grad_fn(learner, push_index) -> device tensor.  Applies eagerly, or T groups at a time."""
+    pulled, counts = {}, {}
+    ready = 0
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == PULL:
+            pulled[l] = ps.pull_weights()
+        else:
+            p = counts.get(l, 0)
+            counts[l] = p + 1
+            ready += ps.push_gradient(l, grad_fn(l, p), pulled[l])
+            if ready and (not lazy or ready >= fuse_t):
+                ready -= ps.apply_update()
+    ps.flush()
+    ps.synchronize()
+
+
+def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, grad_std, kinds, learners,
+             w0: torch.Tensor, seed: int, fuse_t: int = 1, lazy: bool = False, precisions=(32, 64),
+             options=None, misalign: int = 0):
+    """Returns (gpu_w, gpu_v, gpu_log, {precision: (w, v, log)})."""
+    dev = torch.device("cuda", 0)
+    tdt = TORCH_DTYPE[grad_dtype]
+    mod = P.binding.MODULATIONS[modulation]
+    refs = {}
+    for prec in precisions:
+        r = R.ReferencePS(num_params, lam, n, alpha0, momentum, wd, mod, prec)
+        r.set_weights(w0.numpy())
+        refs[prec] = r
+
+    state = None
+    if misalign:                      # state carved out at an odd element offset: scalar kernel path
+        wbuf = torch.zeros(num_params + misalign + 8, dtype=torch.float32, device=dev)
+        vbuf = torch.zeros(num_params + misalign + 8, dtype=torch.float32, device=dev)
+        state = (wbuf[misalign:misalign + num_params], vbuf[misalign:misalign + num_params])
+    ps = P.ParameterServer(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, fuse_t,
+                           device=dev, state=state)
+    for key, val in (options or {}).items():
+        ps.set_option(key, val)
+    ps.init_weights(w0.to(dev))
+
+    def grad_fn(l, p):
+        if misalign:
+            buf = torch.empty(num_params + misalign, dtype=tdt, device=dev)
+            g = buf[misalign:]
+            G.gradient(seed, l, p, num_params, grad_std, dtype=tdt, device=dev, out=g)
+        else:
+            g = G.gradient(seed, l, p, num_params, grad_std, dtype=tdt, device=dev)
+        host = as_reference_grad(g)
+        for r in refs.values():
+            r_fired = r.push(l, host)
+        return g
+
+    # the reference consumes pulls too: interleave by wrapping the replay
+    pulled, counts = {}, {}
+    ready = 0
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == PULL:
+            pulled[l] = ps.pull_weights()
+            for r in refs.values():
+                assert r.pull(l) == pulled[l]          # timestamps agree call by call
+        else:
+            p = counts.get(l, 0)
+            counts[l] = p + 1
+            ready += ps.push_gradient(l, grad_fn(l, p), pulled[l])
+            if ready and (not lazy or ready >= fuse_t):
+                ready -= ps.apply_update()
+    ps.flush()
+    ps.synchronize()
+    out = {prec: (*r.state(), r.log()) for prec, r in refs.items()}
+    w = ps.w[:num_params].cpu().numpy().copy()
+    v = ps.v[:num_params].cpu().numpy().copy()
+    log = ps.update_log()
+    ps.destroy()
+    return w, v, log, out
+
+
+def assert_logs_equal(log, rlog):
+    for f in ("update", "push_index", "ts_grad", "tau", "sigma", "learner", "position"):
+        assert np.array_equal(log[f], rlog[f]), f
+    assert np.array_equal(log["scale"], rlog["scale"].astype(np.float32))
+    assert np.array_equal(log["decay"], rlog["decay"].astype(np.float32))
+
+
+def assert_parity(w, v, log, refs, tol, layout=None):
+    """Bit-exact against the fp32 reference, within `tol` relative L2 against the fp64 one."""
+    if 32 in refs:
+        w32, v32, log32 = refs[32]
+        assert_logs_equal(log, log32)
+        assert np.array_equal(w, w32.astype(np.float32)), "weights differ from the fp32 reference"
+        assert np.array_equal(v, v32.astype(np.float32)), "momentum differs from the fp32 reference"
+    if 64 in refs:
+        w64, v64, log64 = refs[64]
+        worst = max(rel_l2(w, w64), rel_l2(v, v64))
+        if layout is not None:
+            for seg in layout.segments:
+                sl = slice(seg.offset, seg.offset + seg.count)
+                if np.linalg.norm(w64[sl]) > 0:
+                    worst = max(worst, rel_l2(w[sl], w64[sl]))
+                if np.linalg.norm(v64[sl]) > 0:
+                    worst = max(worst, rel_l2(v[sl], v64[sl]))
+        assert worst <= tol, "relative L2 error %.3e above %.1e" % (worst, tol)
+        return worst
+    return 0.0

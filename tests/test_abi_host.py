@@ -1,0 +1,205 @@
+"""C-ABI surface and host-side protocol logic, without a GPU.
+
+A server with zero parameters launches nothing, so its whole state machine
+(timestamps, staleness, grouping, scale table, log, error codes) can be driven
+here and compared field by field with the reference.
+"""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_1511_05950_b200 as P
+from oracle import reference as R
+from tests.helpers import PULL
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+FAKE_GRAD = 0x1000          # never dereferenced: zero-length gradients
+
+
+def declared_symbols():
+    names = []
+    inc = os.path.join(ROOT, "include")
+    for fn in sorted(os.listdir(inc)):
+        if fn.endswith(".h"):
+            text = open(os.path.join(inc, fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names += re.findall(r"^\s*(?:int|const char \*)\s*\*?(ps_\w+)\s*\(", text, flags=re.M)
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_symbols()
+    assert len(names) >= 18 and "ps_apply_update" in names
+    for n in names:
+        assert hasattr(P.lib, n), n
+    assert sorted(names) == sorted(P.binding.EXPORTS)
+
+
+def make(lam, n, alpha0=0.01, m=0.9, wd=5e-4, mod=P.PS_MOD_INV_STALENESS, num_params=0):
+    h = C.c_void_p()
+    rc = P.ps_create(C.byref(h), num_params, lam, n, alpha0, m, wd, mod)
+    return rc, h
+
+
+def drive(h, kinds, learners, fuse_t=1, lazy=False):
+    """Replay a trace; apply as soon as a group completes (or lazily, T at a time)."""
+    assert P.ps_set_option(h, P.PS_OPT_FUSE_T, fuse_t) == 0
+    pulled = {}
+    ts = C.c_int64()
+    ready = 0
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == PULL:
+            assert P.ps_pull_weights(h, None, C.byref(ts)) == 0
+            pulled[l] = ts.value
+        else:
+            rc = P.ps_push_gradient(h, l, FAKE_GRAD, pulled[l])
+            assert rc in (P.PS_OK, P.PS_READY)
+            ready += rc == P.PS_READY
+            if ready and (not lazy or ready == fuse_t):
+                assert P.ps_apply_update(h) == ready
+                ready = 0
+    assert P.ps_flush(h) == ready
+
+
+def fetch_log(h, c):
+    a = C.c_int64()
+    assert P.ps_peek_state(h, None, None, C.byref(a), None) == 0
+    out = np.empty(a.value * c, dtype=P.binding.LOG_DTYPE)
+    assert P.ps_get_update_log(h, 0, a.value, out.ctypes.data) == 0
+    return a.value, out
+
+
+@pytest.mark.parametrize("model,lam,n,mod", [
+    ("rounds", 4, 1, "inv_staleness"), ("exp", 30, 30, "inv_staleness"), ("uniform", 18, 4, "inv_staleness"),
+    ("lognormal", 54, 54, "inv_staleness"), ("exp", 12, 3, "constant"), ("lognormal", 9, 2, "inv_staleness"),
+])
+@pytest.mark.parametrize("fuse_t,lazy", [(1, False), (8, True)])
+def test_schedule_matches_reference_bit_exactly(model, lam, n, mod, fuse_t, lazy):
+    pushes = 600
+    kinds, learners = R.simulate_arrivals(model, lam, pushes, 42)
+    ref = R.ReferencePS(0, lam, n, 0.01, 0.9, 5e-4, P.binding.MODULATIONS[mod], 32)
+    ref.set_weights(np.zeros(0, np.float32))
+    nothing = np.zeros(0, np.float32)
+    counts = {}
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        ref.pull(l) if k == PULL else ref.push(l, nothing)
+    rlog = ref.log()
+
+    rc, h = make(lam, n, mod=P.binding.MODULATIONS[mod])
+    assert rc == 0
+    drive(h, kinds, learners, fuse_t, lazy)
+    c = lam // n
+    ts, log = fetch_log(h, c)
+    assert ts == ref.timestamp == pushes // c
+    for f in ("update", "push_index", "ts_grad", "tau", "sigma", "learner", "position"):
+        assert np.array_equal(log[f], rlog[f]), f
+    assert np.array_equal(log["scale"], rlog["scale"].astype(np.float32))      # fp32 reference: exact widening
+    assert np.array_equal(log["decay"], rlog["decay"].astype(np.float32))
+    assert P.ps_destroy(h) == 0
+
+
+def test_logical_clock_runs_ahead_of_applied_clock():
+    rc, h = make(2, 2)
+    ts, a, l = C.c_int64(), C.c_int64(), C.c_int64()
+    for i in range(5):
+        assert P.ps_pull_weights(h, None, C.byref(ts)) == 0 and ts.value == i
+        assert P.ps_push_gradient(h, 0, FAKE_GRAD, ts.value) == P.PS_READY
+    P.ps_peek_state(h, None, None, C.byref(a), C.byref(l))
+    assert (a.value, l.value) == (0, 5)
+    P.ps_set_option(h, P.PS_OPT_FUSE_T, 3)
+    assert P.ps_apply_update(h) == 3 and P.ps_apply_update(h) == 2
+    assert P.ps_apply_update(h) == P.PS_ERR_NOT_READY
+    P.ps_peek_state(h, None, None, C.byref(a), C.byref(l))
+    assert (a.value, l.value) == (5, 5)
+    P.ps_destroy(h)
+
+
+def test_error_codes():
+    h = C.c_void_p()
+    assert P.ps_create(None, 0, 1, 1, 0.1, 0.0, 0.0, 1) == P.PS_ERR_INVALID_ARG
+    assert P.ps_create(C.byref(h), 0, 3, 4, 0.1, 0.0, 0.0, 1) == P.PS_ERR_INVALID_ARG      # n > lambda
+    assert P.ps_create(C.byref(h), 0, 3, 0, 0.1, 0.0, 0.0, 1) == P.PS_ERR_INVALID_ARG
+    assert P.ps_create(C.byref(h), -1, 3, 1, 0.1, 0.0, 0.0, 1) == P.PS_ERR_INVALID_ARG
+    assert P.ps_create(C.byref(h), 0, 3, 1, 0.1, 0.0, 0.0, 7) == P.PS_ERR_INVALID_ARG      # modulation
+    assert P.ps_create(C.byref(h), 0, 1000, 1, 0.1, 0.0, 0.0, 1) == P.PS_ERR_INVALID_ARG   # c > PS_MAX_GROUP
+    assert P.ps_create(C.byref(h), 0, 3, 1, float("nan"), 0.0, 0.0, 1) == P.PS_ERR_INVALID_ARG
+    rc, h = make(3, 1)
+    assert rc == 0
+    ts = C.c_int64()
+    assert P.ps_pull_weights(h, None, None) == P.PS_ERR_INVALID_ARG
+    assert P.ps_push_gradient(h, 3, FAKE_GRAD, 0) == P.PS_ERR_BAD_LEARNER
+    assert P.ps_push_gradient(h, -1, FAKE_GRAD, 0) == P.PS_ERR_BAD_LEARNER
+    assert P.ps_push_gradient(h, 0, FAKE_GRAD, 1) == P.PS_ERR_BAD_TIMESTAMP       # from the future: tau < 0
+    assert P.ps_push_gradient(h, 0, FAKE_GRAD, -1) == P.PS_ERR_BAD_TIMESTAMP
+    assert P.ps_push_gradient(h, 0, None, 0) == P.PS_ERR_INVALID_ARG
+    assert P.ps_push_gradient(h, 0, FAKE_GRAD + 2, 0) == P.PS_ERR_INVALID_ARG     # fp32 needs 4-byte alignment
+    assert P.ps_push_gradient_host(h, 0, FAKE_GRAD, 0) == P.PS_ERR_NO_STATE       # no staging slots bound
+    assert P.ps_apply_update(h) == P.PS_ERR_NOT_READY
+    assert P.ps_push_gradient(h, 0, FAKE_GRAD, 0) == P.PS_OK
+    assert P.ps_push_gradient(h, 1, FAKE_GRAD, 0) == P.PS_OK
+    assert P.ps_apply_update(h) == P.PS_ERR_NOT_READY                             # 2 of 3 pending
+    assert P.ps_set_option(h, P.PS_OPT_GRAD_DTYPE, P.PS_GRAD_BF16) == P.PS_ERR_INVALID_ARG  # while pending
+    assert P.ps_push_gradient(h, 1, FAKE_GRAD, 0) == P.PS_READY
+    # rejected calls left the state untouched
+    a, l = C.c_int64(), C.c_int64()
+    P.ps_peek_state(h, None, None, C.byref(a), C.byref(l))
+    assert (a.value, l.value) == (0, 1)
+    for key, bad in ((P.PS_OPT_FUSE_T, 0), (P.PS_OPT_FUSE_T, 17), (P.PS_OPT_QUEUE_GROUPS, 0), (P.PS_OPT_KERNEL, 9),
+                     (P.PS_OPT_BLOCK_THREADS, 100), (P.PS_OPT_BLOCK_THREADS, 1024), (99, 1), (P.PS_OPT_GRAD_DTYPE, 5)):
+        assert P.ps_set_option(h, key, bad) == P.PS_ERR_INVALID_ARG
+    assert P.ps_get_update_log(h, 0, 1, None) == P.PS_ERR_INVALID_ARG
+    buf = np.empty(3, dtype=P.binding.LOG_DTYPE)
+    assert P.ps_get_update_log(h, 0, 1, buf.ctypes.data) == P.PS_ERR_LOG_EVICTED   # not applied yet
+    assert P.ps_apply_update(h) == 1
+    assert P.ps_get_update_log(h, 0, 1, buf.ctypes.data) == 0
+    assert buf["learner"].tolist() == [0, 1, 1] and buf["push_index"].tolist() == [0, 0, 1]
+    assert P.ps_destroy(h) == 0
+    assert P.ps_destroy(h) == P.PS_ERR_INVALID_ARG                                 # use after destroy is refused
+    assert P.ps_apply_update(h) == P.PS_ERR_INVALID_ARG
+    assert P.ps_destroy(None) == P.PS_ERR_INVALID_ARG
+
+
+def test_queue_limit_and_log_window():
+    rc, h = make(1, 1)
+    assert P.ps_set_option(h, P.PS_OPT_QUEUE_GROUPS, 4) == 0
+    assert P.ps_set_option(h, P.PS_OPT_LOG_UPDATES, 3) == 0
+    for i in range(4):
+        assert P.ps_push_gradient(h, 0, FAKE_GRAD, i) == P.PS_READY
+    assert P.ps_push_gradient(h, 0, FAKE_GRAD, 4) == P.PS_ERR_QUEUE_FULL
+    assert P.ps_flush(h) == 4
+    assert P.ps_push_gradient(h, 0, FAKE_GRAD, 4) == P.PS_READY
+    assert P.ps_flush(h) == 1
+    buf = np.empty(3, dtype=P.binding.LOG_DTYPE)
+    assert P.ps_get_update_log(h, 1, 3, buf.ctypes.data) == P.PS_ERR_LOG_EVICTED
+    assert P.ps_get_update_log(h, 2, 3, buf.ctypes.data) == 0
+    assert buf["update"].tolist() == [2, 3, 4]
+    P.ps_destroy(h)
+
+
+def test_group_larger_than_one_launch_clamps_fusion():
+    rc, h = make(256, 1)                      # c = 256: at most 2 groups fit PS_MAX_ENTRIES
+    assert rc == 0
+    P.ps_set_option(h, P.PS_OPT_FUSE_T, 16)
+    for g in range(5):
+        for l in range(256):
+            P.ps_push_gradient(h, l, FAKE_GRAD, 0)
+    assert [P.ps_apply_update(h) for _ in range(3)] == [2, 2, 1]
+    P.ps_destroy(h)
+
+
+def test_status_strings():
+    assert P.status_string(P.PS_ERR_BAD_TIMESTAMP).startswith("gradient timestamp")
+    assert P.status_string(0) == "ok"
+
+
+def test_compute_without_a_gpu_fails_loudly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    rc, h = make(2, 1, num_params=1024)
+    assert rc == P.PS_ERR_CUDA and not h.value
+    with pytest.raises(P.SoftsyncError):
+        P.ParameterServer(1024, 2, 1, 0.1, allocate=False)

@@ -1,0 +1,54 @@
+"""The N > 1 path of bench.py on CPU: two gloo ranks, replicas only (no data-path collective)."""
+import os
+import socket
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import bench
+from workloads import configs
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    mine = [10.0 + rank, 3.0 - rank, 1.0]
+    got = bench.max_over_ranks(mine, torch.device("cpu"), world)
+    dist.barrier()
+    out.put((rank, got))
+    dist.destroy_process_group()
+
+
+def test_timings_are_reduced_with_max_over_two_gloo_ranks():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    results = dict(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert results[0] == results[1] == [11.0, 3.0, 1.0]
+
+
+def test_whole_job_value_counts_every_replica():
+    one = bench.whole_job_value(1, 1000, 10, 5.0)
+    assert bench.whole_job_value(4, 1000, 10, 5.0) == 4 * one == 4 * 1000 * 10 / 5e-3
+
+
+def test_steps_group_trace_events_by_completed_update():
+    cfg = configs.LARGE_SOFTSYNC
+    steps = bench.step_events(cfg, 25)
+    assert len(steps) == 25
+    for evs in steps:
+        assert sum(k == 1 for k, _ in evs) == cfg.c and evs[-1][0] == 1
+    assert bench.algorithmic_bytes(60965224, 4, 4) == 60965224 * 32

@@ -1,0 +1,108 @@
+"""Parity at the benchmark's full sizes, on sampled elements.
+
+The update is element-wise, so the reference can follow any subset of elements on its own:
+the GPU runs the whole 60,965,224-element vector through the default launch configuration
+(the one bench.py times), gradients generated on the device; the reference runs the same
+protocol on a few thousand sampled elements whose inputs the generator reproduces bit for
+bit on the CPU.  Timestamps, staleness and grouping do not depend on the vector length and
+are compared in full.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_1511_05950_b200 as P
+from oracle import reference as R
+from tests.gpu_harness import TORCH_DTYPE, as_reference_grad, assert_logs_equal
+from tests.helpers import PULL, rel_l2
+from workloads import configs, generators as G
+
+pytestmark = pytest.mark.gpu
+
+
+def sample_indices(layout, count, seed):
+    n = layout.num_params
+    rng = np.random.default_rng(seed)
+    idx = set(rng.integers(0, n, size=count).tolist())
+    for seg in layout.segments:                       # every layer boundary, both sides
+        for k in range(-8, 8):
+            for base in (seg.offset, seg.offset + seg.count):
+                if 0 <= base + k < n:
+                    idx.add(base + k)
+    idx.update(range(0, 64))
+    idx.update(range(n - 64, n))
+    return torch.tensor(sorted(idx), dtype=torch.int64)
+
+
+def run_full(cfg, lazy, num_pushes=None):
+    dev = torch.device("cuda", 0)
+    layout = cfg.layout()
+    n = layout.num_params
+    pushes = num_pushes or cfg.num_pushes
+    tdt = TORCH_DTYPE[cfg.grad_dtype]
+    idx = sample_indices(layout, 6000, 1)
+    idx_dev = idx.to(dev)
+    kinds, learners = R.simulate_arrivals(cfg.arrival_model, cfg.num_learners, pushes, cfg.seed)
+
+    refs = {}
+    w0_s = G.initial_weights_at(layout, cfg.seed, idx, cfg.weight_std)
+    for prec in (32, 64):
+        r = R.ReferencePS(idx.numel(), cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
+                          P.binding.MODULATIONS[cfg.modulation], prec)
+        r.set_weights(w0_s.numpy())
+        refs[prec] = r
+
+    ps = P.ParameterServer(n, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
+                           cfg.modulation, cfg.grad_dtype, cfg.fuse_t, device=dev)
+    ps.init_weights(G.initial_weights(layout, cfg.seed, cfg.weight_std, device=dev))
+    assert torch.equal(ps.w[idx_dev].cpu(), w0_s)      # same generator bits on both devices
+
+    pulled, counts, ready = {}, {}, 0
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == PULL:
+            pulled[l] = ps.pull_weights()
+            for r in refs.values():
+                assert r.pull(l) == pulled[l]
+            continue
+        p = counts.get(l, 0)
+        counts[l] = p + 1
+        g = G.gradient(cfg.seed, l, p, n, cfg.grad_std, dtype=tdt, device=dev)
+        gs = G.gradient_at(cfg.seed, l, p, idx, cfg.grad_std, dtype=tdt)
+        if p == 0:
+            assert torch.equal(g[idx_dev].cpu(), gs)
+        host = as_reference_grad(gs)
+        for r in refs.values():
+            r.push(l, host)
+        ready += ps.push_gradient(l, g, pulled[l])
+        if ready and (not lazy or ready >= cfg.fuse_t):
+            ready -= ps.apply_update()
+    ps.flush()
+    ps.synchronize()
+
+    w = ps.w[idx_dev].cpu().numpy()
+    v = ps.v[idx_dev].cpu().numpy()
+    log = ps.update_log()
+    assert ps.timestamps() == (pushes // cfg.c, pushes // cfg.c)
+    assert torch.isfinite(ps.w).all() and torch.isfinite(ps.v).all()
+    ps.destroy()
+
+    w32, v32 = refs[32].state()
+    assert_logs_equal(log, refs[32].log())
+    assert np.array_equal(w, w32.astype(np.float32)) and np.array_equal(v, v32.astype(np.float32))
+    w64, v64 = refs[64].state()
+    tol = 1e-3 if cfg.grad_dtype == "bf16" else 1e-5
+    assert rel_l2(w, w64) <= tol and rel_l2(v, v64) <= tol
+    return log
+
+
+def test_large_softsync_full_size():
+    """Config 3: 60,965,224 elements, lambda=18, n=4 (c=4), fp32 gradients, 500 updates."""
+    log = run_full(configs.LARGE_SOFTSYNC, lazy=False)
+    assert log["update"][-1] == 499
+    assert 3.0 < log["tau"][200:].mean() < 5.5          # <tau> close to n = 4 (Section 2.4)
+
+
+def test_large_stale_bf16_full_size():
+    """Config 4: same vector, lambda=54, n=54 (c=1), bf16 gradients, 2,000 pushes applied 8 per pass."""
+    log = run_full(configs.LARGE_STALE_BF16, lazy=True)
+    assert len(log) == 2000 and log["tau"].max() > 100

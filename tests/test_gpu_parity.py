@@ -1,0 +1,216 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU reference, element by element.
+
+Tolerances: the benchmark's — relative L2 <= 1e-5 on final weights and momentum against the
+fp64 reference (<= 1e-3 with bf16 gradients) — and, stricter, bit equality with the fp32
+reference, because the kernel performs the same separately rounded fp32 operations in the
+same order.  Timestamps, staleness and group membership must be bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_1511_05950_b200 as P
+from oracle import reference as R
+from tests.gpu_harness import run_pair, assert_parity
+from workloads import configs, generators as G, layouts
+
+pytestmark = pytest.mark.gpu
+
+TOL_FP32 = 1e-5
+TOL_BF16 = 1e-3
+
+
+def run_config(cfg, num_pushes=None, layout=None, **kw):
+    layout = layout or cfg.layout()
+    pushes = num_pushes or cfg.num_pushes
+    kinds, learners = R.simulate_arrivals(cfg.arrival_model, cfg.num_learners, pushes, cfg.seed)
+    w0 = G.initial_weights(layout, cfg.seed, cfg.weight_std)
+    w, v, log, refs = run_pair(layout.num_params, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum,
+                               cfg.weight_decay, cfg.modulation, cfg.grad_dtype, cfg.grad_std,
+                               kinds, learners, w0, cfg.seed, **kw)
+    tol = TOL_BF16 if cfg.grad_dtype == "bf16" else TOL_FP32
+    worst = assert_parity(w, v, log, refs, tol, layout)
+    return worst, log
+
+
+def test_tiny_softsync_full():
+    """Config 1 in full: lambda=4, n=1, 89,578 elements, 200 updates."""
+    cfg = configs.TINY_SOFTSYNC
+    worst, log = run_config(cfg)
+    assert log["update"][-1] == 199 and (log["sigma"] == 1).all()
+
+
+def test_pure_async_full():
+    """Config 2 in full: lambda=30, n=30, 10,000 pushes with Exp(1) compute times."""
+    cfg = configs.PURE_ASYNC
+    worst, log = run_config(cfg)
+    assert len(log) == 10000 and log["sigma"].max() > 60
+
+
+def test_large_softsync_scaled_down():
+    """Config 3's protocol (lambda=18, n=4, uniform arrivals) on a ragged vector of several tiles."""
+    cfg = configs.LARGE_SOFTSYNC
+    run_config(cfg, num_pushes=600, layout=layouts.flat(5 * 65536 + 4099))
+
+
+@pytest.mark.parametrize("lazy", [False, True])
+def test_large_stale_bf16_scaled_down(lazy):
+    """Config 4's protocol (lambda=54, n=54, bf16 gradients, T=8) on a ragged vector."""
+    cfg = configs.LARGE_STALE_BF16
+    worst, log = run_config(cfg, num_pushes=400, layout=layouts.flat(3 * 65536 + 2053), fuse_t=8, lazy=lazy)
+    assert log["sigma"].max() > 20
+
+
+def _simple(num_params, lam, n, pushes, grad_dtype="fp32", model="exp", seed=77, **kw):
+    kinds, learners = R.simulate_arrivals(model, lam, pushes, seed)
+    w0 = G.initial_weights(layouts.flat(num_params), seed) if num_params else torch.zeros(0)
+    w, v, log, refs = run_pair(num_params, lam, n, 0.01, 0.9, 5e-4, "inv_staleness", grad_dtype, 1e-3,
+                               kinds, learners, w0, seed, **kw)
+    assert_parity(w, v, log, refs, TOL_BF16 if grad_dtype == "bf16" else TOL_FP32)
+    return w, v, log
+
+
+@pytest.mark.parametrize("grad_dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("num_params", [1, 2, 3, 4, 5, 7, 8, 9, 15, 16, 17, 31, 33, 1023, 1025,
+                                        16384, 16385, 16386, 16387, 16388, 16389, 16390, 16391])
+def test_ragged_sizes(num_params, grad_dtype):
+    _simple(num_params, 6, 3, 24, grad_dtype)
+
+
+@pytest.mark.parametrize("grad_dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("misalign", [1, 2, 3])
+def test_pointers_not_16_byte_aligned_take_the_scalar_path(misalign, grad_dtype):
+    _simple(10007, 5, 2, 30, grad_dtype, misalign=misalign)
+
+
+@pytest.mark.parametrize("grad_dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("lam,n", [(1, 1), (2, 1), (3, 1), (7, 1), (8, 1), (9, 1), (16, 1), (17, 1), (64, 1), (100, 1), (256, 1)])
+def test_group_sizes(lam, n, grad_dtype):
+    _simple(4099, lam, n, 3 * lam, grad_dtype, model="uniform")
+
+
+@pytest.mark.parametrize("grad_dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("fuse_t", [2, 3, 8, 16])
+@pytest.mark.parametrize("lam,n", [(4, 4), (6, 2), (40, 2)])
+def test_temporal_fusion_is_invisible(lam, n, fuse_t, grad_dtype):
+    """T groups per pass give the same bits as one group per pass."""
+    pushes = 20 * (lam // n) + (lam // n) // 2
+    a = _simple(8 * 1024 + 5, lam, n, pushes, grad_dtype, model="lognormal", fuse_t=fuse_t, lazy=True)
+    b = _simple(8 * 1024 + 5, lam, n, pushes, grad_dtype, model="lognormal", fuse_t=1, lazy=False)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    assert np.array_equal(a[2], b[2])
+
+
+@pytest.mark.parametrize("options", [
+    {P.PS_OPT_KERNEL: P.PS_KERNEL_SCALAR}, {P.PS_OPT_KERNEL: P.PS_KERNEL_VECTOR},
+    {P.PS_OPT_GRID_BLOCKS: 1}, {P.PS_OPT_GRID_BLOCKS: 7, P.PS_OPT_BLOCK_THREADS: 128},
+    {P.PS_OPT_BLOCK_THREADS: 512}, {P.PS_OPT_GRID_BLOCKS: 148 * 3, P.PS_OPT_BLOCK_THREADS: 512},
+])
+def test_launch_shape_does_not_change_the_bits(options):
+    _simple(70001, 8, 2, 40, "fp32", options=options)
+    _simple(70001, 8, 2, 40, "bf16", options=options)
+
+
+def test_zero_parameters():
+    _simple(0, 4, 2, 12)
+
+
+def test_constant_modulation_and_plain_rule():
+    kinds, learners = R.simulate_arrivals("exp", 10, 60, 5)
+    w0 = G.initial_weights(layouts.flat(5000), 5)
+    for mod, m, wd in (("constant", 0.9, 5e-4), ("inv_staleness", 0.0, 0.0)):
+        w, v, log, refs = run_pair(5000, 10, 5, 0.02, m, wd, mod, "fp32", 1e-3, kinds, learners, w0, 5)
+        assert_parity(w, v, log, refs, TOL_FP32)
+
+
+def test_guard_bands_stay_untouched():
+    """State and gradients sit between poisoned guard regions; nothing outside [0, N) is written,
+    and gradients are never written at all."""
+    dev = torch.device("cuda", 0)
+    for grad_dtype, tdt in (("fp32", torch.float32), ("bf16", torch.bfloat16)):
+        for n_el in (16384 + 3, 999):
+            pad = 1024
+            wbuf = torch.full((n_el + 2 * pad,), 7.25, device=dev)
+            vbuf = torch.full((n_el + 2 * pad,), -3.5, device=dev)
+            ps = P.ParameterServer(n_el, 3, 1, 0.01, 0.9, 5e-4, grad_dtype=grad_dtype, device=dev,
+                                   state=(wbuf[pad:pad + n_el], vbuf[pad:pad + n_el]))
+            ps.init_weights(G.initial_weights(layouts.flat(n_el), 3).to(dev))
+            grads = []
+            for l in range(3):
+                gb = torch.full((n_el + 2 * pad,), 1.5, dtype=tdt, device=dev)
+                G.gradient(3, l, 0, n_el, 1e-3, dtype=tdt, device=dev, out=gb[pad:pad + n_el])
+                grads.append((gb, gb.clone()))
+                ps.push_gradient(l, gb[pad:pad + n_el], ps.pull_weights())
+            assert ps.apply_update() == 1
+            ps.synchronize()
+            for buf, val in ((wbuf, 7.25), (vbuf, -3.5)):
+                assert (buf[:pad] == val).all() and (buf[pad + n_el:] == val).all()
+            for gb, before in grads:
+                assert torch.equal(gb, before)
+            ps.destroy()
+
+
+def test_weight_pull_flushes_pending_groups_and_host_paths():
+    """A pull that returns weights applies every complete group first; host push/pull agree with device ones."""
+    dev = torch.device("cuda", 0)
+    n_el, lam = 30011, 4
+    w0 = G.initial_weights(layouts.flat(n_el), 9)
+    results = []
+    for host in (False, True):
+        ps = P.ParameterServer(n_el, lam, 2, 0.01, 0.9, 5e-4, fuse_t=4, device=dev)
+        ps.init_weights(w0 if host else w0.to(dev))
+        if host:
+            ps.bind_staging(2 * 3)
+        ts = {l: ps.pull_weights() for l in range(lam)}
+        for p in range(3):
+            for l in range(2):
+                g = G.gradient(9, l, p, n_el, 1e-3, device="cpu" if host else dev)
+                if host:
+                    g = g.pin_memory()
+                ps.push_gradient(l, g, ts[l])
+        assert ps.timestamps() == (0, 3)
+        out = torch.empty(n_el, device="cpu" if host else dev)
+        assert ps.pull_weights(out) == 3
+        assert ps.timestamps() == (3, 3)
+        ps.synchronize()
+        results.append(out.cpu().numpy().copy())
+        assert np.array_equal(results[-1], ps.w.cpu().numpy())
+        ps.destroy()
+    assert np.array_equal(results[0], results[1])
+    ref = R.ReferencePS(n_el, lam, 2, 0.01, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    for l in range(lam):
+        ref.pull(l)
+    for p in range(3):
+        for l in range(2):
+            ref.push(l, G.gradient(9, l, p, n_el, 1e-3).numpy())
+    assert np.array_equal(results[0], ref.state()[0].astype(np.float32))
+
+
+def test_staging_slots_run_out():
+    dev = torch.device("cuda", 0)
+    ps = P.ParameterServer(64, 4, 1, 0.01, device=dev)
+    ps.init_weights(torch.zeros(64))
+    ps.bind_staging(2)
+    g = torch.ones(64)
+    ps.push_gradient(0, g, 0)
+    ps.push_gradient(1, g, 0)
+    with pytest.raises(P.SoftsyncError) as e:
+        ps.push_gradient(2, g, 0)
+    assert e.value.status == P.PS_ERR_QUEUE_FULL
+    ps.destroy()
+
+
+def test_kernel_timing_option_counts_launches():
+    dev = torch.device("cuda", 0)
+    ps = P.ParameterServer(1 << 16, 1, 1, 0.01, device=dev)
+    ps.init_weights(torch.zeros(1 << 16))
+    ps.set_option(P.PS_OPT_TIMING, 1)
+    g = torch.ones(1 << 16, device=dev)
+    for i in range(5):
+        ps.push_gradient(0, g, i)
+        ps.apply_update()
+    ms, launches = ps.kernel_time()
+    assert launches == 5 and ms > 0
+    assert ps.kernel_time() == (0.0, 0)
+    ps.destroy()

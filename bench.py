@@ -200,51 +200,53 @@ def run_ours(args, cfg, rank, world, local_rank):
     for s in range(args.warmup):
         one_step(ev_steps, s, pool)
     ps.synchronize()
-    ps.set_option(P.PS_OPT_TIMING, 1)
-    ps.kernel_time()
+    applied_before = ps.timestamps()[0]
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     with ClockSampler(local_rank) as clocks:
-        start.record()
+        start.record()                             # torch's current stream is the server's stream
         for s in range(args.warmup, total_steps):
             one_step(ev_steps, s, pool)
         stop.record()
         torch.cuda.synchronize(dev)
     barrier()
     elapsed_ms = start.elapsed_time(stop)
-    kernel_ms, launches = ps.kernel_time()
-    ps.set_option(P.PS_OPT_TIMING, 0)
+    # one update kernel per step and nothing else on the stream between the two events
+    launches = (ps.timestamps()[0] - applied_before) // groups_per_step
     assert launches == args.steps
+    kernel_ms = elapsed_ms
 
-    # ---- end to end: gradients from pinned host memory, updated weights back to the host
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    host_pool = [torch.empty(n, dtype=tdt).pin_memory() for _ in range(min(4, pool_n))]
-    for hb, db in zip(host_pool, pool):
-        hb.copy_(db)
-    w_host = torch.empty(n, dtype=torch.float32).pin_memory()
-    ps.bind_staging(2 * cfg.c * fuse_t)
-    ps.init_weights(G.initial_weights(layout, cfg.seed + rank, cfg.weight_std, device=dev))
-    pulled.clear()
-    e2e_events = step_events(cfg, (1 + e2e_steps) * groups_per_step)
+    e2e_steps, e2e_s = 0, 0.0
+    if not args.no_e2e:
+        # ---- end to end: gradients from pinned host memory, updated weights back to the host
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        host_pool = [torch.empty(n, dtype=tdt).pin_memory() for _ in range(min(4, pool_n))]
+        for hb, db in zip(host_pool, pool):
+            hb.copy_(db)
+        w_host = torch.empty(n, dtype=torch.float32).pin_memory()
+        ps.bind_staging(2 * cfg.c * fuse_t)
+        ps.init_weights(G.initial_weights(layout, cfg.seed + rank, cfg.weight_std, device=dev))
+        pulled.clear()
+        e2e_events = step_events(cfg, (1 + e2e_steps) * groups_per_step)
 
-    def e2e_step(s):
-        one_step(e2e_events, s, host_pool)
-        ps.pull_weights(w_host)                    # device -> host read of the step's result (synchronous)
+        def e2e_step(s):
+            one_step(e2e_events, s, host_pool)
+            ps.pull_weights(w_host)                    # device -> host read of the step's result (synchronous)
 
-    e2e_step(0)
-    barrier()
-    t0 = time.perf_counter()
-    for s in range(1, 1 + e2e_steps):
-        e2e_step(s)
-    torch.cuda.synchronize(dev)
-    e2e_s = time.perf_counter() - t0
-    barrier()
+        e2e_step(0)
+        barrier()
+        t0 = time.perf_counter()
+        for s in range(1, 1 + e2e_steps):
+            e2e_step(s)
+        torch.cuda.synchronize(dev)
+        e2e_s = time.perf_counter() - t0
+        barrier()
 
     elapsed_ms, e2e_ms, kern_ms = max_over_ranks([elapsed_ms, e2e_s * 1e3, kernel_ms / max(1, launches)], dev, world)
 
     elems_per_step = cfg.c * n * groups_per_step
     value = whole_job_value(world, elems_per_step, args.steps, elapsed_ms)
-    e2e_value = whole_job_value(world, elems_per_step, e2e_steps, e2e_ms)
+    e2e_value = whole_job_value(world, elems_per_step, e2e_steps, e2e_ms) if e2e_steps else None
     abytes = algorithmic_bytes(n, cfg.c * fuse_t, gbytes)
     peak, peak_kind = hbm_peak()
     achieved = abytes / (kern_ms * 1e-3) / 1e9
@@ -268,10 +270,12 @@ def run_ours(args, cfg, rank, world, local_rank):
         "clocks": clocks.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
                 "h2d_bytes_per_step": cfg.c * fuse_t * n * gbytes, "d2h_bytes_per_step": n * 4,
-                "ms_per_step": e2e_ms / e2e_steps},
+                "ms_per_step": e2e_ms / e2e_steps if e2e_steps else None},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": TRAFFIC.get(cfg.name), "of": peak_kind,
-                     "kernel_ms": kern_ms, "algorithmic_bytes": abytes},
+                     "kernel_ms": kern_ms, "algorithmic_bytes": abytes,
+                     "how": "CUDA events around the %d back-to-back launches of the timed region / %d "
+                            "(inter-launch gaps included)" % (args.steps, args.steps)},
     }
     ps.destroy()
     return result
@@ -342,6 +346,70 @@ def run_reference(args, cfg):
     }
 
 
+def run_sweep(args):
+    """Bandwidth sweep: flat fp32 vectors of 1M .. 1B parameters, c in {1,4,16,64}, fp32 and bf16
+    gradients, staleness uniform in [1, 2c], 50 updates per point after 5 warm-up updates."""
+    import paper_1511_05950_b200 as P
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = hbm_peak()
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+    rng = np.random.default_rng(configs.SEED)
+    points = []
+    updates, warm = 50, 5
+    for n in configs.SWEEP_SIZES:
+        for grad_dtype, tdt, gb in (("fp32", torch.float32, 4), ("bf16", torch.bfloat16, 2)):
+            for c in configs.SWEEP_C:
+                abytes = algorithmic_bytes(n, c, gb)
+                pool_n = max(c, min(64, -(-(4 * l2_bytes) // (n * gb))))
+                need = n * 8 + pool_n * n * gb + (2 << 30)
+                torch.cuda.empty_cache()
+                free, _ = torch.cuda.mem_get_info(dev)
+                point = {"num_params": n, "c": c, "grad_dtype": grad_dtype, "algorithmic_bytes": abytes,
+                         "fits_l2": bool(abytes <= l2_bytes)}
+                if need > free:
+                    point["skipped"] = "does not fit: needs %.1f GB, %.1f GB free" % (need / 1e9, free / 1e9)
+                    points.append(point)
+                    continue
+                ps = P.ParameterServer(n, c, 1, 0.01, 0.9, 5e-4, "inv_staleness", grad_dtype, 1, device=dev)
+                ps.set_option(P.PS_OPT_QUEUE_GROUPS, 4)
+                w0 = torch.empty(n, dtype=torch.float32, device=dev)
+                G.normal_like(G.stream_key(configs.SEED, G.STREAM_WEIGHTS), 0, n, 0.01, out=w0)
+                ps.init_weights(w0)
+                del w0
+                pool = []
+                for i in range(pool_n):
+                    buf = torch.empty(n, dtype=tdt, device=dev)
+                    G.gradient(configs.SEED, i, 0, n, 1e-4, dtype=tdt, device=dev, out=buf)
+                    pool.append(buf)
+                k = 0
+                start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                for u in range(warm + updates):
+                    if u == warm:
+                        torch.cuda.synchronize(dev)
+                        start.record()
+                    now = ps.pull_weights()
+                    for l in range(c):
+                        sigma = int(rng.integers(1, 2 * c + 1))
+                        ps.push_gradient(l, pool[k % pool_n], max(0, now - sigma))
+                        k += 1
+                    ps.apply_update()
+                stop.record()
+                torch.cuda.synchronize(dev)
+                ms = start.elapsed_time(stop) / updates
+                point.update({"us_per_update": ms * 1e3, "gbs": abytes / ms / 1e6, "frac_of_%s_copy_peak" % peak_kind:
+                              abytes / ms / 1e6 / peak, "grad_elements_per_s": c * n / (ms * 1e-3)})
+                points.append(point)
+                ps.destroy()
+                del pool
+                print("N=%-11d %s c=%-3d %9.1f us  %7.1f GB/s  %5.1f%% of %s copy peak%s" % (
+                    n, grad_dtype, c, ms * 1e3, point["gbs"], 100 * point["gbs"] / peak, peak_kind,
+                    "  (fits L2: not an HBM figure)" if point["fits_l2"] else ""), file=sys.stderr, flush=True)
+    return {"metric": "hbm_gbs_per_softsync_update", "unit": "GB/s", "peak": peak, "of": peak_kind,
+            "updates_per_point": updates, "warmup": warm, "sweep": points}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -351,9 +419,18 @@ def main():
     ap.add_argument("--workload", default="large_softsync", choices=sorted(configs.BY_NAME))
     ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
+    ap.add_argument("--num-params", type=int, default=0,
+                    help="run the workload's protocol on a flat vector of this many parameters (profiler captures)")
+    ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over sizes, group sizes and gradient types")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     cfg = configs.BY_NAME[args.workload]
+    if args.num_params:
+        from dataclasses import replace
+        from workloads import layouts
+        flat_n = args.num_params
+        cfg = replace(cfg, name="%s@flat%d" % (cfg.name, flat_n), layout=lambda: layouts.flat(flat_n))
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -362,6 +439,10 @@ def main():
     if args.impl == "reference":
         if rank == 0:
             print(json.dumps(run_reference(args, cfg)), flush=True)
+        return
+    if args.sweep:
+        if rank == 0:
+            print(json.dumps(run_sweep(args)), flush=True)
         return
 
     if world > 1:

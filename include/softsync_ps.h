@@ -59,8 +59,7 @@ enum ps_option {
     PS_OPT_LOG_UPDATES = 5,               /* how many most recent updates the log keeps (default 65536) */
     PS_OPT_TIMING = 6,                    /* 1: bracket every update kernel with CUDA events (ps_kernel_time) */
     PS_OPT_KERNEL = 7,                    /* ps_kernel_choice (default PS_KERNEL_AUTO) */
-    PS_OPT_GRID_BLOCKS = 8,               /* thread blocks per launch; 0 = chosen from the SM count */
-    PS_OPT_BLOCK_THREADS = 9              /* threads per block: 128, 256 or 512; 0 = default */
+    PS_OPT_BLOCK_THREADS = 8              /* threads per block: 128, 256 or 512; 0 = default (128) */
 };
 
 enum ps_kernel_choice {

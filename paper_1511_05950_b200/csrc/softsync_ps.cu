@@ -48,7 +48,7 @@ struct ps_ctx {
     cudaStream_t stream = nullptr;
     int64_t queue_groups = 64;
     int64_t log_updates = 65536;
-    int timing = 0, kernel_choice = PS_KERNEL_AUTO, grid_blocks = 0, block_threads = 0;
+    int timing = 0, kernel_choice = PS_KERNEL_AUTO, block_threads = 0;
     int sm_count = 0;
 
     int64_t ts_applied = 0;                // updates whose kernel has been enqueued
@@ -94,11 +94,34 @@ bool entry_before(const Entry &a, const Entry &b)
     return a.learner != b.learner ? a.learner < b.learner : a.push_index < b.push_index;
 }
 
-template <typename GT, int VEC, int K, int MAXE>
+constexpr int kChunk = 8;            // gradient loads in flight per thread beyond the first EC
+constexpr int kHeadFp32 = 16;        // largest compile-time first chunk, fp32 gradients
+constexpr int kHeadBf16 = 8;         // same for bf16 gradients
+
+template <typename GT, int VEC, int EC, bool MORE, int MAXE>
 cudaError_t launch_variant(const LaunchParams<MAXE> &p, int blocks, int threads, cudaStream_t stream)
 {
-    softsync::softsync_update_kernel<GT, VEC, K, MAXE><<<blocks, threads, 0, stream>>>(p);
+    softsync::softsync_update_kernel<GT, VEC, EC, MORE, kChunk, MAXE><<<blocks, threads, 0, stream>>>(p);
     return cudaGetLastError();
+}
+
+// E = T*c <= HEAD: the straight-line instantiation with exactly E loads up front.
+template <typename GT, int VEC, int HEAD, int MAXE, int EC = HEAD>
+cudaError_t launch_exact(int E, const LaunchParams<MAXE> &p, int blocks, int threads, cudaStream_t stream)
+{
+    if constexpr (EC == 0) {
+        return cudaErrorInvalidValue;
+    } else {
+        if (E == EC) return launch_variant<GT, VEC, EC, false, MAXE>(p, blocks, threads, stream);
+        return launch_exact<GT, VEC, HEAD, MAXE, EC - 1>(E, p, blocks, threads, stream);
+    }
+}
+
+template <typename GT, int VEC, int HEAD, int MAXE>
+cudaError_t launch_vector(int E, const LaunchParams<MAXE> &p, int blocks, int threads, cudaStream_t stream)
+{
+    if (E <= HEAD) return launch_exact<GT, VEC, (HEAD < MAXE ? HEAD : MAXE), MAXE>(E, p, blocks, threads, stream);
+    return launch_variant<GT, VEC, HEAD, true, MAXE>(p, blocks, threads, stream);   // HEAD loads, then chunks
 }
 
 template <int MAXE>
@@ -106,18 +129,17 @@ cudaError_t launch_update(ps_ctx *ps, const LaunchParams<MAXE> &p, bool vector_o
 {
     const bool bf16 = ps->grad_dtype == PS_GRAD_BF16;
     const int vec = vector_ok ? (bf16 ? 8 : 4) : 1;
-    const int threads = ps->block_threads ? ps->block_threads : 256;
+    const int threads = ps->block_threads ? ps->block_threads : 128;
     const long long frags = std::max<long long>(1, (p.n + vec - 1) / vec);
-    long long blocks = (frags + threads - 1) / threads;
-    const long long cap = ps->grid_blocks ? ps->grid_blocks
-                                          : static_cast<long long>(ps->sm_count) * (2048 / threads) * 4;
-    blocks = std::max<long long>(1, std::min(blocks, cap));
+    const long long blocks = (frags + threads - 1) / threads;    // one fragment per thread
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     const int b = static_cast<int>(blocks);
-    if (vector_ok)
-        return bf16 ? launch_variant<GradBf16, 8, 8, MAXE>(p, b, threads, ps->stream)
-                    : launch_variant<GradFp32, 4, 8, MAXE>(p, b, threads, ps->stream);
-    return bf16 ? launch_variant<GradBf16, 1, 8, MAXE>(p, b, threads, ps->stream)
-                : launch_variant<GradFp32, 1, 8, MAXE>(p, b, threads, ps->stream);
+    const int E = p.T * p.c;
+    if (!vector_ok)
+        return bf16 ? launch_variant<GradBf16, 1, 0, true, MAXE>(p, b, threads, ps->stream)
+                    : launch_variant<GradFp32, 1, 0, true, MAXE>(p, b, threads, ps->stream);
+    return bf16 ? launch_vector<GradBf16, 8, kHeadBf16, MAXE>(E, p, b, threads, ps->stream)
+                : launch_vector<GradFp32, 4, kHeadFp32, MAXE>(E, p, b, threads, ps->stream);
 }
 
 // Fills the scale table of one launch (Eq. 3 folded with the 1/c of Eq. 2) for the `T`
@@ -239,7 +261,7 @@ int push_common(ps_ctx *ps, int learner, const void *grad_dev, int64_t ts, int s
 
 int check_push(ps_ctx *ps, int learner, const void *grad, int64_t ts)
 {
-    if (!grad) return PS_ERR_INVALID_ARG;
+    if (!grad && ps->n > 0) return PS_ERR_INVALID_ARG;    // a zero-length gradient has no address
     if (learner < 0 || learner >= ps->lambda) return PS_ERR_BAD_LEARNER;
     if (ts < 0 || ts > ts_logical(ps)) return PS_ERR_BAD_TIMESTAMP;
     if (static_cast<int64_t>(ps->ready.size()) >= ps->queue_groups) return PS_ERR_QUEUE_FULL;
@@ -315,8 +337,8 @@ int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev)
 
 int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host)
 {
-    if (!is_live(ps) || !w_src) return PS_ERR_INVALID_ARG;
-    if (!ps->w || !ps->v) return PS_ERR_NO_STATE;
+    if (!is_live(ps) || (!w_src && ps->n > 0)) return PS_ERR_INVALID_ARG;
+    if (ps->n > 0 && (!ps->w || !ps->v)) return PS_ERR_NO_STATE;
     const size_t bytes = static_cast<size_t>(ps->n) * sizeof(float);
     if (bytes) {
         PS_CUDA(ps, cudaMemcpyAsync(ps->w, w_src, bytes, src_is_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, ps->stream));
@@ -372,9 +394,6 @@ int ps_set_option(ps_t *ps, int key, int64_t value)
     case PS_OPT_KERNEL:
         if (value < PS_KERNEL_AUTO || value > PS_KERNEL_VECTOR) return PS_ERR_INVALID_ARG;
         ps->kernel_choice = static_cast<int>(value); return PS_OK;
-    case PS_OPT_GRID_BLOCKS:
-        if (value < 0 || value > 0x7fffffff) return PS_ERR_INVALID_ARG;
-        ps->grid_blocks = static_cast<int>(value); return PS_OK;
     case PS_OPT_BLOCK_THREADS:
         if (value != 0 && value != 128 && value != 256 && value != 512) return PS_ERR_INVALID_ARG;
         ps->block_threads = static_cast<int>(value); return PS_OK;
@@ -394,7 +413,6 @@ int ps_get_option(ps_t *ps, int key, int64_t *value)
     case PS_OPT_LOG_UPDATES: *value = ps->log_updates; return PS_OK;
     case PS_OPT_TIMING: *value = ps->timing; return PS_OK;
     case PS_OPT_KERNEL: *value = ps->kernel_choice; return PS_OK;
-    case PS_OPT_GRID_BLOCKS: *value = ps->grid_blocks; return PS_OK;
     case PS_OPT_BLOCK_THREADS: *value = ps->block_threads; return PS_OK;
     default: return PS_ERR_INVALID_ARG;
     }

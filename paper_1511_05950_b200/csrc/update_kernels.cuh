@@ -1,10 +1,10 @@
 // Fused sumGradients + applyUpdate kernels of the n-softsync parameter server
 // (arXiv 1511.05950, Section 2.1; Eq. 2 with the per-gradient rate of Eq. 3).
 //
-// One pass over the parameter vector: every thread owns VEC consecutive
-// elements, loads theta and v once, streams the T*c gradient values of those
-// elements through registers, applies the T updates in order and stores theta
-// and v once.  The path is HBM-bound (about 0.3 flop per byte), so the work is
+// One pass over the parameter vector: every thread owns one fragment of VEC
+// consecutive elements, loads theta and v once, streams the T*c gradient values
+// of those elements through registers, applies the T updates in order and
+// stores theta and v once.  The path is HBM-bound (about 0.3 flop per byte), so the work is
 // plain fp32 ALU code around wide coalesced loads; tensor cores have no part.
 //
 // Arithmetic contract (bit-exact, any launch shape): per element and per group
@@ -113,65 +113,93 @@ __device__ __forceinline__ void store_state(float *p, const float (&x)[VEC])
     }
 }
 
-// ---- VEC elements starting at element index first = i * VEC ----------------
-template <typename GT, int VEC, int K, int MAXE>
-__device__ __forceinline__ void update_fragment(const LaunchParams<MAXE> &p, long long i, long long first)
-{
+// ---- running state of one fragment while its gradients stream through -------
+template <int VEC>
+struct Fragment {
     float w[VEC], v[VEC], acc[VEC];
-    load_state<VEC>(p.w + first, w);
-    load_state<VEC>(p.v + first, v);
-    const int E = p.T * p.c;
-    const float m = p.momentum;
-    int l = 0, t = 0;
-    for (int e0 = 0; e0 < E; e0 += K) {
-        Raw<GT, VEC> raw[K];
+    int l, t;                         // position inside the current group, group index
+};
+
+// Adds gradient entry e (already in registers) to the fragment; when it is the
+// last of its group, performs that group's weight update.  Branches are uniform
+// across the grid (they depend on e and c only).
+template <typename GT, int VEC, int MAXE>
+__device__ __forceinline__ void consume(const LaunchParams<MAXE> &p, Fragment<VEC> &f, const Raw<GT, VEC> &r, int e)
+{
+    float g[VEC];
+    widen(r, g);
+    const float s = p.s[e];
+    if (f.l == 0) {
 #pragma unroll
-        for (int k = 0; k < K; ++k)                      // K independent loads in flight
-            if (e0 + k < E) load_raw(raw[k], p.g[e0 + k], i);
+        for (int j = 0; j < VEC; ++j) f.acc[j] = __fmul_rn(s, g[j]);
+    } else {
 #pragma unroll
-        for (int k = 0; k < K; ++k) {
-            if (e0 + k < E) {
-                float g[VEC];
-                widen(raw[k], g);
-                const float s = p.s[e0 + k];
-                if (l == 0) {
+        for (int j = 0; j < VEC; ++j) f.acc[j] = __fadd_rn(f.acc[j], __fmul_rn(s, g[j]));
+    }
+    if (++f.l == p.c) {                                  // group complete: one weight update
+        const float d = p.d[f.t++];
+        const float m = p.momentum;
+        f.l = 0;
 #pragma unroll
-                    for (int j = 0; j < VEC; ++j) acc[j] = __fmul_rn(s, g[j]);
-                } else {
-#pragma unroll
-                    for (int j = 0; j < VEC; ++j) acc[j] = __fadd_rn(acc[j], __fmul_rn(s, g[j]));
-                }
-                if (++l == p.c) {                        // group complete: one weight update
-                    const float d = p.d[t++];
-                    l = 0;
-#pragma unroll
-                    for (int j = 0; j < VEC; ++j) {
-                        const float tt = __fadd_rn(acc[j], __fmul_rn(d, w[j]));
-                        v[j] = __fadd_rn(__fmul_rn(m, v[j]), tt);
-                        w[j] = __fsub_rn(w[j], v[j]);
-                    }
-                }
-            }
+        for (int j = 0; j < VEC; ++j) {
+            const float tt = __fadd_rn(f.acc[j], __fmul_rn(d, f.w[j]));
+            f.v[j] = __fadd_rn(__fmul_rn(m, f.v[j]), tt);
+            f.w[j] = __fsub_rn(f.w[j], f.v[j]);
         }
     }
-    store_state<VEC>(p.w + first, w);
-    store_state<VEC>(p.v + first, v);
 }
 
-// Grid-stride over fragments of VEC elements; the (n mod VEC) trailing
-// elements are done one by one by the first threads of the grid.
-template <typename GT, int VEC, int K, int MAXE>
+// VEC elements starting at element `first` (fragment index i).  The first EC
+// gradient loads and the theta/v loads are issued back to back before anything
+// is consumed, so every thread has (EC + 2) independent 16-byte requests in
+// flight.  MORE = false: the launch has exactly EC entries and the code is
+// straight-line (no spare registers held for a loop that never runs).
+// MORE = true: entries beyond EC follow in chunks of K loads.
+template <typename GT, int VEC, int EC, bool MORE, int K, int MAXE>
+__device__ __forceinline__ void update_fragment(const LaunchParams<MAXE> &p, long long i, long long first)
+{
+    Fragment<VEC> f;
+    Raw<GT, VEC> head[EC > 0 ? EC : 1];
+#pragma unroll
+    for (int e = 0; e < EC; ++e) load_raw(head[e], p.g[e], i);
+    load_state<VEC>(p.w + first, f.w);
+    load_state<VEC>(p.v + first, f.v);
+    f.l = 0; f.t = 0;
+#pragma unroll
+    for (int e = 0; e < EC; ++e) consume<GT, VEC, MAXE>(p, f, head[e], e);
+    if constexpr (MORE) {
+        const int E = p.T * p.c;
+        for (int e0 = EC; e0 < E; e0 += K) {
+            Raw<GT, VEC> raw[K];
+#pragma unroll
+            for (int k = 0; k < K; ++k)
+                if (e0 + k < E) load_raw(raw[k], p.g[e0 + k], i);
+#pragma unroll
+            for (int k = 0; k < K; ++k)
+                if (e0 + k < E) consume<GT, VEC, MAXE>(p, f, raw[k], e0 + k);
+        }
+    }
+    store_state<VEC>(p.w + first, f.w);
+    store_state<VEC>(p.v + first, f.v);
+}
+
+// One fragment of VEC elements per thread: the grid covers the vector exactly once
+// (blocks * threads >= n / VEC).  No grid-stride loop: a loop around the fragment
+// makes the compiler keep a second iteration's registers alive and costs a third
+// of the occupancy.  The host guarantees T*c == EC (MORE = false) or T*c > EC
+// (MORE = true).  The (n mod VEC) trailing elements are done one by one by the
+// first threads of the grid.
+template <typename GT, int VEC, int EC, bool MORE, int K, int MAXE>
 __global__ void softsync_update_kernel(const __grid_constant__ LaunchParams<MAXE> p)
 {
     const long long nfrag = p.n / VEC;
     const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-    for (long long i = tid; i < nfrag; i += stride)
-        update_fragment<GT, VEC, K, MAXE>(p, i, i * VEC);
+    if (tid < nfrag)
+        update_fragment<GT, VEC, EC, MORE, K, MAXE>(p, tid, tid * VEC);
     if constexpr (VEC > 1) {
         const long long done = nfrag * VEC;
         if (tid < p.n - done)
-            update_fragment<GT, 1, K, MAXE>(p, done + tid, done + tid);
+            update_fragment<GT, 1, 0, true, K, MAXE>(p, done + tid, done + tid);
     }
 }
 

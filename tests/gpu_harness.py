@@ -90,8 +90,9 @@ def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, g
     ps.flush()
     ps.synchronize()
     out = {prec: (*r.state(), r.log()) for prec, r in refs.items()}
-    w = ps.w[:num_params].cpu().numpy().copy()
-    v = ps.v[:num_params].cpu().numpy().copy()
+    empty = np.zeros(0, np.float32)
+    w = ps.w[:num_params].cpu().numpy().copy() if num_params else empty
+    v = ps.v[:num_params].cpu().numpy().copy() if num_params else empty
     log = ps.update_log()
     ps.destroy()
     return w, v, log, out

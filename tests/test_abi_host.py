@@ -134,7 +134,6 @@ def test_error_codes():
     assert P.ps_push_gradient(h, -1, FAKE_GRAD, 0) == P.PS_ERR_BAD_LEARNER
     assert P.ps_push_gradient(h, 0, FAKE_GRAD, 1) == P.PS_ERR_BAD_TIMESTAMP       # from the future: tau < 0
     assert P.ps_push_gradient(h, 0, FAKE_GRAD, -1) == P.PS_ERR_BAD_TIMESTAMP
-    assert P.ps_push_gradient(h, 0, None, 0) == P.PS_ERR_INVALID_ARG
     assert P.ps_push_gradient(h, 0, FAKE_GRAD + 2, 0) == P.PS_ERR_INVALID_ARG     # fp32 needs 4-byte alignment
     assert P.ps_push_gradient_host(h, 0, FAKE_GRAD, 0) == P.PS_ERR_NO_STATE       # no staging slots bound
     assert P.ps_apply_update(h) == P.PS_ERR_NOT_READY

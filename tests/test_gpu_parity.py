@@ -103,8 +103,8 @@ def test_temporal_fusion_is_invisible(lam, n, fuse_t, grad_dtype):
 
 @pytest.mark.parametrize("options", [
     {P.PS_OPT_KERNEL: P.PS_KERNEL_SCALAR}, {P.PS_OPT_KERNEL: P.PS_KERNEL_VECTOR},
-    {P.PS_OPT_GRID_BLOCKS: 1}, {P.PS_OPT_GRID_BLOCKS: 7, P.PS_OPT_BLOCK_THREADS: 128},
-    {P.PS_OPT_BLOCK_THREADS: 512}, {P.PS_OPT_GRID_BLOCKS: 148 * 3, P.PS_OPT_BLOCK_THREADS: 512},
+    {P.PS_OPT_BLOCK_THREADS: 128}, {P.PS_OPT_BLOCK_THREADS: 256}, {P.PS_OPT_BLOCK_THREADS: 512},
+    {P.PS_OPT_KERNEL: P.PS_KERNEL_SCALAR, P.PS_OPT_BLOCK_THREADS: 512},
 ])
 def test_launch_shape_does_not_change_the_bits(options):
     _simple(70001, 8, 2, 40, "fp32", options=options)
@@ -185,6 +185,17 @@ def test_weight_pull_flushes_pending_groups_and_host_paths():
         for l in range(2):
             ref.push(l, G.gradient(9, l, p, n_el, 1e-3).numpy())
     assert np.array_equal(results[0], ref.state()[0].astype(np.float32))
+
+
+def test_null_and_misaligned_gradient_pointers_are_rejected():
+    import ctypes as C
+    dev = torch.device("cuda", 0)
+    ps = P.ParameterServer(64, 2, 1, 0.01, device=dev)
+    assert P.ps_push_gradient(ps._h, 0, None, 0) == P.PS_ERR_INVALID_ARG
+    g = torch.ones(66, device=dev)
+    assert P.ps_push_gradient(ps._h, 0, g.data_ptr() + 2, 0) == P.PS_ERR_INVALID_ARG
+    assert ps.timestamps() == (0, 0)
+    ps.destroy()
 
 
 def test_staging_slots_run_out():

@@ -111,6 +111,46 @@ def test_launch_shape_does_not_change_the_bits(options):
     _simple(70001, 8, 2, 40, "bf16", options=options)
 
 
+@pytest.mark.parametrize("grad_dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("c", [1, 4, 16, 64])
+def test_sweep_point_with_uniform_staleness(c, grad_dtype):
+    """The bandwidth sweep's smallest size (2^20 flat elements): c gradients per update, each with a
+    staleness drawn uniformly from [1, 2c] (learners push with an old timestamp)."""
+    dev = torch.device("cuda", 0)
+    n_el, updates = 1 << 20, 6
+    tdt = torch.bfloat16 if grad_dtype == "bf16" else torch.float32
+    rng = np.random.default_rng(c)
+    w0 = G.initial_weights(layouts.flat(n_el), 11)
+    ps = P.ParameterServer(n_el, c, 1, 0.01, 0.9, 5e-4, "inv_staleness", grad_dtype, device=dev)
+    ps.init_weights(w0.to(dev))
+    w, v = w0.numpy().astype(np.float32), np.zeros(n_el, np.float32)
+    m, a0, wd = np.float32(0.9), np.float64(np.float32(0.01)), np.float64(np.float32(5e-4))
+    for u in range(updates):
+        now = ps.pull_weights()
+        assert now == u
+        sig = []
+        acc = None
+        for l in range(c):
+            sigma = int(rng.integers(1, 2 * c + 1))
+            ts = max(0, now - sigma)
+            g = G.gradient(11, l, u, n_el, 1e-4, dtype=tdt, device=dev)
+            ps.push_gradient(l, g, ts)
+            eff = max(now - ts, 1)
+            sig.append(eff)
+            s = np.float32(a0 / (np.float64(c) * eff))
+            term = s * g.float().cpu().numpy()
+            acc = term if acc is None else acc + term
+        assert ps.apply_update() == 1
+        d = np.float32(wd * sum(np.float64(np.float32(a0 / (np.float64(c) * e))) for e in sig))
+        v = m * v + (acc + d * w)
+        w = w - v
+        log = ps.update_log(u, 1)
+        assert log["sigma"].tolist() == sig and (log["tau"] == np.minimum(now, log["tau"])).all()
+    ps.synchronize()
+    assert np.array_equal(ps.w.cpu().numpy(), w) and np.array_equal(ps.v.cpu().numpy(), v)
+    ps.destroy()
+
+
 def test_zero_parameters():
     _simple(0, 4, 2, 12)
 

@@ -7,7 +7,7 @@ from __future__ import annotations
 
 import contextlib
 import ctypes as C
-from typing import Tuple
+from typing import Optional, Tuple
 
 import numpy as np
 
@@ -44,6 +44,7 @@ def load(path: str) -> C.CDLL:
         L.oracle_ps_pull.restype = C.c_int64
         L.oracle_ps_pull.argtypes = [C.c_void_p, C.c_int]
         L.oracle_ps_push.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int]
+        L.oracle_ps_push_with_timestamp.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int64]
         L.oracle_ps_get_state.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.oracle_ps_log_size.restype = C.c_int64
         L.oracle_ps_log_size.argtypes = [C.c_void_p]
@@ -120,8 +121,9 @@ class ReferencePS:
             raise ValueError("bad learner id")
         return ts
 
-    def push(self, learner: int, grad: np.ndarray) -> bool:
-        """grad: float32 values, or uint16 holding bf16 bit patterns."""
+    def push(self, learner: int, grad: np.ndarray, timestamp: Optional[int] = None) -> bool:
+        """grad: float32 values, or uint16 holding bf16 bit patterns.  timestamp: the clock value the
+        gradient carries; by default the one this learner pulled last."""
         grad = np.ascontiguousarray(grad)
         assert grad.size == self.num_params
         if grad.dtype == np.float32:
@@ -130,7 +132,10 @@ class ReferencePS:
             kind = GRAD_BF16
         else:
             raise TypeError("gradient must be float32 or uint16 (bf16 bits)")
-        r = lib().oracle_ps_push(self._h, learner, grad.ctypes.data, kind)
+        if timestamp is None:
+            r = lib().oracle_ps_push(self._h, learner, grad.ctypes.data, kind)
+        else:
+            r = lib().oracle_ps_push_with_timestamp(self._h, learner, grad.ctypes.data, kind, timestamp)
         if r < 0:
             raise ValueError("oracle_ps_push failed with %d" % r)
         return bool(r)

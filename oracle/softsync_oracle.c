@@ -201,13 +201,14 @@ static void apply_pending(oracle_ps *ps)
     ps->npending = 0;
 }
 
-/* pushGradient + sumGradients (+ applyUpdate when the group is complete).
+/* pushGradient + sumGradients (+ applyUpdate when the group is complete), with the gradient's
+ * timestamp j given by the caller: "a learner pushes gradient with timestamp j to the parameter
+ * server of timestamp i, where i >= j" (Section 2.1).
  * Returns 1 if this push triggered a weight update, 0 if not, < 0 on misuse. */
-int oracle_ps_push(oracle_ps *ps, int learner, const void *grad, int grad_dtype)
+int oracle_ps_push_with_timestamp(oracle_ps *ps, int learner, const void *grad, int grad_dtype, int64_t j)
 {
     if (learner < 0 || learner >= ps->lambda) return -1;
-    const int64_t j = ps->pulled_ts[learner];
-    if (j < 0) return -2;                                /* pushed before ever pulling */
+    if (j < 0) return -2;
     const int64_t tau = ps->ts - j;                      /* staleness, Section 2.1 */
     if (tau < 0) return -3;
     int64_t sigma = 1;
@@ -224,6 +225,13 @@ int oracle_ps_push(oracle_ps *ps, int learner, const void *grad, int grad_dtype)
     }
     if (ps->npending == ps->c) { apply_pending(ps); return 1; }
     return 0;
+}
+
+/* The usual case: the gradient carries the timestamp of the learner's latest pull (Section 2.1). */
+int oracle_ps_push(oracle_ps *ps, int learner, const void *grad, int grad_dtype)
+{
+    if (learner < 0 || learner >= ps->lambda) return -1;
+    return oracle_ps_push_with_timestamp(ps, learner, grad, grad_dtype, ps->pulled_ts[learner]);
 }
 
 void oracle_ps_get_state(const oracle_ps *ps, double *w_out, double *v_out)

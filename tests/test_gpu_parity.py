@@ -114,8 +114,9 @@ def test_launch_shape_does_not_change_the_bits(options):
 @pytest.mark.parametrize("grad_dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("c", [1, 4, 16, 64])
 def test_sweep_point_with_uniform_staleness(c, grad_dtype):
-    """The bandwidth sweep's smallest size (2^20 flat elements): c gradients per update, each with a
-    staleness drawn uniformly from [1, 2c] (learners push with an old timestamp)."""
+    """The bandwidth sweep's smallest size (2^20 flat elements): c gradients per update, each pushed with
+    a timestamp that makes its staleness uniform in [1, 2c] (clamped while the clock is still young)."""
+    from tests.gpu_harness import as_reference_grad, assert_logs_equal
     dev = torch.device("cuda", 0)
     n_el, updates = 1 << 20, 6
     tdt = torch.bfloat16 if grad_dtype == "bf16" else torch.float32
@@ -123,32 +124,25 @@ def test_sweep_point_with_uniform_staleness(c, grad_dtype):
     w0 = G.initial_weights(layouts.flat(n_el), 11)
     ps = P.ParameterServer(n_el, c, 1, 0.01, 0.9, 5e-4, "inv_staleness", grad_dtype, device=dev)
     ps.init_weights(w0.to(dev))
-    w, v = w0.numpy().astype(np.float32), np.zeros(n_el, np.float32)
-    m, a0, wd = np.float32(0.9), np.float64(np.float32(0.01)), np.float64(np.float32(5e-4))
+    refs = {prec: R.ReferencePS(n_el, c, 1, 0.01, 0.9, 5e-4, R.MOD_INV_STALENESS, prec) for prec in (32, 64)}
+    for r in refs.values():
+        r.set_weights(w0.numpy())
     for u in range(updates):
         now = ps.pull_weights()
-        assert now == u
-        sig = []
-        acc = None
+        assert now == u == refs[32].timestamp
         for l in range(c):
-            sigma = int(rng.integers(1, 2 * c + 1))
-            ts = max(0, now - sigma)
+            ts = max(0, now - int(rng.integers(1, 2 * c + 1)))
             g = G.gradient(11, l, u, n_el, 1e-4, dtype=tdt, device=dev)
             ps.push_gradient(l, g, ts)
-            eff = max(now - ts, 1)
-            sig.append(eff)
-            s = np.float32(a0 / (np.float64(c) * eff))
-            term = s * g.float().cpu().numpy()
-            acc = term if acc is None else acc + term
+            for r in refs.values():
+                r.push(l, as_reference_grad(g), timestamp=ts)
         assert ps.apply_update() == 1
-        d = np.float32(wd * sum(np.float64(np.float32(a0 / (np.float64(c) * e))) for e in sig))
-        v = m * v + (acc + d * w)
-        w = w - v
-        log = ps.update_log(u, 1)
-        assert log["sigma"].tolist() == sig and (log["tau"] == np.minimum(now, log["tau"])).all()
     ps.synchronize()
-    assert np.array_equal(ps.w.cpu().numpy(), w) and np.array_equal(ps.v.cpu().numpy(), v)
+    w, v, log = ps.w.cpu().numpy(), ps.v.cpu().numpy(), ps.update_log()
     ps.destroy()
+    out = {prec: (*r.state(), r.log()) for prec, r in refs.items()}
+    assert_parity(w, v, log, out, TOL_BF16 if grad_dtype == "bf16" else TOL_FP32)
+    assert log["sigma"].max() > 1 or c == 1
 
 
 def test_zero_parameters():

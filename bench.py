@@ -231,13 +231,16 @@ def run_ours(args, cfg, rank, world, local_rank):
 
         def e2e_step(s):
             one_step(e2e_events, s, host_pool)
-            ps.pull_weights(w_host)                    # device -> host read of the step's result (synchronous)
+            ps.pull_weights(w_host, non_blocking=True)  # device -> host read of the step's result, overlapped
+                                                        # with the next step's host -> device gradient copies
 
         e2e_step(0)
+        ps.synchronize()
         barrier()
         t0 = time.perf_counter()
         for s in range(1, 1 + e2e_steps):
             e2e_step(s)
+        ps.synchronize()                               # every read-back has landed in host memory
         torch.cuda.synchronize(dev)
         e2e_s = time.perf_counter() - t0
         barrier()

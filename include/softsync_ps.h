@@ -121,6 +121,14 @@ int ps_pull_weights(ps_t *ps, float *out_dev, int64_t *ts);
 /* Same, into host memory; returns after the copy has completed. */
 int ps_pull_weights_host(ps_t *ps, float *out_host, int64_t *ts);
 
+/* Same, but returns as soon as the copy is enqueued on a second, library-owned stream, so that it
+ * overlaps host-to-device gradient copies issued afterwards (full-duplex PCIe).  The copy waits for
+ * the updates enqueued so far; later updates wait for the copy before they overwrite theta.
+ * out_host should be pinned memory and must not be read before ps_synchronize (or a later
+ * ps_pull_weights_host) has returned.  The paper's learners block in pullWeights (Section 2.3);
+ * this is the non-blocking form of the same call. */
+int ps_pull_weights_host_async(ps_t *ps, float *out_host, int64_t *ts);
+
 /* pushGradient + the bookkeeping half of sumGradients (Section 2.1, 2.2).  grad_dev: num_params
  * values of the configured dtype, BORROWED: it must stay valid and unchanged until the
  * ps_apply_update that consumes it has finished on the stream.  ts: the timestamp the learner
@@ -150,7 +158,7 @@ int ps_apply_update(ps_t *ps);
 /* Applies every complete pending group (repeated ps_apply_update).  Returns the number applied (>= 0). */
 int ps_flush(ps_t *ps);
 
-/* Blocks until the stream has finished everything this handle enqueued. */
+/* Blocks until everything this handle enqueued (main stream and read-back stream) has finished. */
 int ps_synchronize(ps_t *ps);
 
 /* Copies the log entries of updates [first_update, first_update + count) to out_host

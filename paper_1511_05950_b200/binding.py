@@ -39,7 +39,7 @@ LOG_DTYPE = np.dtype([
 
 EXPORTS = (
     "ps_create", "ps_destroy", "ps_bind_state", "ps_init_weights", "ps_bind_staging",
-    "ps_set_option", "ps_get_option", "ps_pull_weights", "ps_pull_weights_host",
+    "ps_set_option", "ps_get_option", "ps_pull_weights", "ps_pull_weights_host", "ps_pull_weights_host_async",
     "ps_push_gradient", "ps_push_gradient_host", "ps_apply_update", "ps_flush", "ps_synchronize",
     "ps_get_update_log", "ps_peek_state", "ps_kernel_time", "ps_last_cuda_error", "ps_status_string",
 )
@@ -69,6 +69,7 @@ def _load() -> C.CDLL:
         "ps_get_option": [vp, i32, C.POINTER(i64)],
         "ps_pull_weights": [vp, vp, C.POINTER(i64)],
         "ps_pull_weights_host": [vp, vp, C.POINTER(i64)],
+        "ps_pull_weights_host_async": [vp, vp, C.POINTER(i64)],
         "ps_push_gradient": [vp, i32, vp, i64],
         "ps_push_gradient_host": [vp, i32, vp, i64],
         "ps_apply_update": [vp],
@@ -100,6 +101,7 @@ ps_set_option = lib.ps_set_option
 ps_get_option = lib.ps_get_option
 ps_pull_weights = lib.ps_pull_weights
 ps_pull_weights_host = lib.ps_pull_weights_host
+ps_pull_weights_host_async = lib.ps_pull_weights_host_async
 ps_push_gradient = lib.ps_push_gradient
 ps_push_gradient_host = lib.ps_push_gradient_host
 ps_apply_update = lib.ps_apply_update
@@ -142,6 +144,7 @@ class ParameterServer:
         self.c = num_learners // n if n >= 1 else 0
         self.grad_dtype = grad_dtype
         self._held = collections.deque()
+        self._host_held = []          # pinned host gradients whose upload may still be in flight
         self._staging = None
         self.w = self.v = None
         if device is None and (allocate or state is not None) and num_params > 0:
@@ -204,12 +207,16 @@ class ParameterServer:
         return out.value
 
     # -- the protocol ----------------------------------------------------------
-    def pull_weights(self, out: Optional[torch.Tensor] = None) -> int:
-        """Timestamp a gradient computed from now on must carry; fills `out` with the weights if given."""
+    def pull_weights(self, out: Optional[torch.Tensor] = None, non_blocking: bool = False) -> int:
+        """Timestamp a gradient computed from now on must carry; fills `out` with the weights if given.
+        non_blocking (host `out` only): return once the copy is enqueued; call synchronize() before reading."""
         ts = C.c_int64()
         if out is not None and not out.is_cuda:
             assert out.dtype == torch.float32 and out.is_contiguous()
-            _check(ps_pull_weights_host(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host")
+            if non_blocking:
+                _check(ps_pull_weights_host_async(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host_async")
+            else:
+                _check(ps_pull_weights_host(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host")
             self._held.clear()
         else:
             _check(ps_pull_weights(self._h, _ptr(out), C.byref(ts)), "ps_pull_weights")
@@ -225,6 +232,9 @@ class ParameterServer:
         else:
             r = _check(ps_push_gradient_host(self._h, learner, grad.data_ptr(), ts), "ps_push_gradient_host")
             self._held.append(None)
+            self._host_held.append(grad)
+            if len(self._host_held) > 1024:
+                self.synchronize()
         return r == PS_READY
 
     def apply_update(self) -> int:
@@ -241,6 +251,7 @@ class ParameterServer:
 
     def synchronize(self) -> None:
         _check(ps_synchronize(self._h), "ps_synchronize")
+        self._host_held.clear()
 
     # -- inspection -------------------------------------------------------------
     def timestamps(self) -> Tuple[int, int]:

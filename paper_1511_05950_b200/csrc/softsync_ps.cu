@@ -61,6 +61,12 @@ struct ps_ctx {
 
     std::vector<TimedLaunch> timed, spare_events;
     int last_cuda_error = 0;
+
+    // asynchronous weight read-back: a second stream so that a device-to-host copy of theta can run
+    // while the next gradients are still arriving host-to-device on the main stream
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t weights_ready = nullptr, weights_copied = nullptr;
+    bool copy_in_flight = false;
 };
 
 namespace {
@@ -178,6 +184,16 @@ void build_launch(ps_ctx *ps, int T, LaunchParams<MAXE> &p, std::vector<ps_log_e
     }
 }
 
+// theta may not be overwritten while an asynchronous read-back is still reading it.
+int order_after_readback(ps_ctx *ps)
+{
+    if (ps->copy_in_flight) {
+        PS_CUDA(ps, cudaStreamWaitEvent(ps->stream, ps->weights_copied, 0));
+        ps->copy_in_flight = false;
+    }
+    return PS_OK;
+}
+
 int take_events(ps_ctx *ps, TimedLaunch &tl)
 {
     if (!ps->spare_events.empty()) { tl = ps->spare_events.back(); ps->spare_events.pop_back(); return PS_OK; }
@@ -198,6 +214,8 @@ int apply_groups(ps_ctx *ps, int T)
     if (ps->kernel_choice == PS_KERNEL_VECTOR && !vector_ok) return PS_ERR_INVALID_ARG;
 
     if (ps->n > 0) {
+        const int rb = order_after_readback(ps);
+        if (rb != PS_OK) return rb;
         TimedLaunch tl{};
         const bool timed = ps->timing && ps->timed.size() < kMaxTimedLaunches;
         if (timed) {
@@ -320,6 +338,11 @@ int ps_destroy(ps_t *ps)
         if (!ps || !g_live.erase(ps)) return PS_ERR_INVALID_ARG;
     }
     if (ps->device >= 0) cudaStreamSynchronize(ps->stream);
+    if (ps->copy_stream) {
+        cudaStreamSynchronize(ps->copy_stream);
+        cudaEventDestroy(ps->weights_ready); cudaEventDestroy(ps->weights_copied);
+        cudaStreamDestroy(ps->copy_stream);
+    }
     release_events(ps);
     for (auto &tl : ps->spare_events) { cudaEventDestroy(tl.start); cudaEventDestroy(tl.stop); }
     delete ps;
@@ -341,6 +364,8 @@ int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host)
     if (ps->n > 0 && (!ps->w || !ps->v)) return PS_ERR_NO_STATE;
     const size_t bytes = static_cast<size_t>(ps->n) * sizeof(float);
     if (bytes) {
+        const int rb = order_after_readback(ps);
+        if (rb != PS_OK) return rb;
         PS_CUDA(ps, cudaMemcpyAsync(ps->w, w_src, bytes, src_is_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, ps->stream));
         PS_CUDA(ps, cudaMemsetAsync(ps->v, 0, bytes, ps->stream));
         if (src_is_host) PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
@@ -463,6 +488,29 @@ int ps_pull_weights_host(ps_t *ps, float *out_host, int64_t *ts)
     return PS_OK;
 }
 
+int ps_pull_weights_host_async(ps_t *ps, float *out_host, int64_t *ts)
+{
+    if (!is_live(ps) || !ts || !out_host) return PS_ERR_INVALID_ARG;
+    if (!ps->w || !ps->v) return PS_ERR_NO_STATE;
+    const int r = ps_flush(ps);
+    if (r < 0) return r;
+    if (!ps->copy_stream) {
+        PS_CUDA(ps, cudaStreamCreateWithFlags(&ps->copy_stream, cudaStreamNonBlocking));
+        PS_CUDA(ps, cudaEventCreateWithFlags(&ps->weights_ready, cudaEventDisableTiming));
+        PS_CUDA(ps, cudaEventCreateWithFlags(&ps->weights_copied, cudaEventDisableTiming));
+    }
+    if (ps->n) {
+        PS_CUDA(ps, cudaEventRecord(ps->weights_ready, ps->stream));
+        PS_CUDA(ps, cudaStreamWaitEvent(ps->copy_stream, ps->weights_ready, 0));
+        PS_CUDA(ps, cudaMemcpyAsync(out_host, ps->w, static_cast<size_t>(ps->n) * sizeof(float),
+                                    cudaMemcpyDeviceToHost, ps->copy_stream));
+        PS_CUDA(ps, cudaEventRecord(ps->weights_copied, ps->copy_stream));
+        ps->copy_in_flight = true;
+    }
+    *ts = ts_logical(ps);
+    return PS_OK;
+}
+
 int ps_push_gradient(ps_t *ps, int learner, const void *grad_dev, int64_t ts)
 {
     if (!is_live(ps)) return PS_ERR_INVALID_ARG;
@@ -491,6 +539,7 @@ int ps_synchronize(ps_t *ps)
 {
     if (!is_live(ps)) return PS_ERR_INVALID_ARG;
     PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+    if (ps->copy_stream) PS_CUDA(ps, cudaStreamSynchronize(ps->copy_stream));
     return PS_OK;
 }
 

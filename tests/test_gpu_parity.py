@@ -232,6 +232,30 @@ def test_null_and_misaligned_gradient_pointers_are_rejected():
     ps.destroy()
 
 
+def test_asynchronous_host_pull_orders_with_later_updates():
+    """The non-blocking read-back returns the weights of its own timestamp even when more updates
+    are enqueued right behind it."""
+    dev = torch.device("cuda", 0)
+    n_el = 3_000_017
+    ps = P.ParameterServer(n_el, 1, 1, 0.05, 0.9, 5e-4, device=dev)
+    ps.init_weights(G.initial_weights(layouts.flat(n_el), 4).to(dev))
+    ps.bind_staging(4)
+    snaps, expect = [], []
+    for step in range(4):
+        g = G.gradient(4, 0, step, n_el, 1e-3).pin_memory()
+        ps.push_gradient(0, g, ps.pull_weights())
+        ps.apply_update()
+        expect.append(ps.w.clone())                     # stream-ordered device copy of theta_{step+1}
+        out = torch.empty(n_el).pin_memory()
+        assert ps.pull_weights(out, non_blocking=True) == step + 1
+        snaps.append(out)
+    ps.synchronize()
+    for out, want in zip(snaps, expect):
+        assert torch.equal(out, want.cpu())
+    assert not torch.equal(snaps[0], snaps[3])
+    ps.destroy()
+
+
 def test_staging_slots_run_out():
     dev = torch.device("cuda", 0)
     ps = P.ParameterServer(64, 4, 1, 0.01, device=dev)

@@ -112,6 +112,11 @@ int ps_bind_staging(ps_t *ps, void *slots_dev, int64_t slot_bytes, int num_slots
 int ps_set_option(ps_t *ps, int key, int64_t value);
 int ps_get_option(ps_t *ps, int key, int64_t *value);
 
+/* Learning-rate schedule (Section 4.3 lowers alpha0 in steps during training): sets the base rate for
+ * gradients pushed from now on.  Gradients already pushed keep the rate that was in force when they
+ * arrived (Section 2.4 sets the rate "for an incoming gradient"). */
+int ps_set_alpha0(ps_t *ps, float alpha0);
+
 /* pullWeights (Section 2.1): *ts receives the server timestamp i a gradient computed on these
  * weights must carry.  If out_dev != NULL, every complete pending group is applied first and
  * theta_i (num_params fp32) is copied to out_dev on the stream, so the weights always belong to
@@ -150,7 +155,8 @@ int ps_push_gradient_host(ps_t *ps, int learner, const void *grad_host, int64_t 
  *     acc = s_1 g_1 + s_2 g_2 + ... + s_c g_c     (ascending learner id, then push index)
  *     v   = momentum * v + (acc + d * theta)
  *     theta = theta - v
- * with s_l = alpha0 / (c * sigma_l) and d = weight_decay * sum_l s_l.  Advances the applied
+ * with s_l = alpha0 / (c * sigma_l), alpha0 as it was when gradient l was pushed, and
+ * d = weight_decay * sum_l s_l.  Advances the applied
  * timestamp by the number of groups and appends to the log.  Returns that number (>= 1) or
  * PS_ERR_NOT_READY. */
 int ps_apply_update(ps_t *ps);

@@ -26,6 +26,9 @@
  *   - the update runs inside the push that completes the group; a pull that
  *     follows sees the new clock.
  *   - momentum and weight decay: see update_rule.inc.
+ *   - the base rate alpha0 may be changed between calls (the step schedules of
+ *     Section 4.3); a gradient is scaled with the alpha0 in force when it arrived,
+ *     since Section 2.4 sets the rate "for an incoming gradient".
  *
  * Parity pins: tests/test_oracle_*.py (hand-worked examples under
  * tests/golden/, closed forms, reductions to plain SGD, invariants).
@@ -77,6 +80,7 @@ typedef struct {
 typedef struct {
     int32_t learner;
     int64_t push_index, ts_grad, tau, sigma;
+    double alpha0;       /* base rate in force at arrival */
     void *grad;          /* N values widened to the working precision */
 } pending_t;
 
@@ -135,6 +139,9 @@ void oracle_ps_set_weights(oracle_ps *ps, const float *w0)
     ps->ts = 0;
 }
 
+/* Learning-rate schedule: the base rate for gradients that arrive from now on (Section 4.3). */
+void oracle_ps_set_alpha0(oracle_ps *ps, float alpha0) { ps->alpha0 = alpha0; }
+
 int64_t oracle_ps_timestamp(const oracle_ps *ps) { return ps->ts; }
 int oracle_ps_group_size(const oracle_ps *ps) { return ps->c; }
 
@@ -180,16 +187,19 @@ static void apply_pending(oracle_ps *ps)
     }
     const void *grads[ORACLE_MAX_C];
     int64_t sigma[ORACLE_MAX_C];
-    double scale[ORACLE_MAX_C];
-    for (int l = 0; l < c; ++l) { grads[l] = ps->pending[order[l]].grad; sigma[l] = ps->pending[order[l]].sigma; }
+    double scale[ORACLE_MAX_C], alpha0[ORACLE_MAX_C];
+    for (int l = 0; l < c; ++l) {
+        grads[l] = ps->pending[order[l]].grad; sigma[l] = ps->pending[order[l]].sigma;
+        alpha0[l] = ps->pending[order[l]].alpha0;
+    }
 
     double d;
     if (ps->precision == 32)
         d = apply_group_f32(ps->w, ps->v, ps->N, c, (const float *const *)grads, sigma,
-                            ps->alpha0, ps->momentum, ps->wd, scale);
+                            alpha0, ps->momentum, ps->wd, scale);
     else
         d = apply_group_f64(ps->w, ps->v, ps->N, c, (const double *const *)grads, sigma,
-                            ps->alpha0, ps->momentum, ps->wd, scale);
+                            alpha0, ps->momentum, ps->wd, scale);
 
     for (int l = 0; l < c; ++l) {
         const pending_t *p = &ps->pending[order[l]];
@@ -217,7 +227,7 @@ int oracle_ps_push_with_timestamp(oracle_ps *ps, int learner, const void *grad, 
 
     pending_t *p = &ps->pending[ps->npending++];
     p->learner = learner; p->push_index = ps->push_count[learner]++;
-    p->ts_grad = j; p->tau = tau; p->sigma = sigma;
+    p->ts_grad = j; p->tau = tau; p->sigma = sigma; p->alpha0 = ps->alpha0;
     for (int64_t k = 0; k < ps->N; ++k) {
         const float g = grad_dtype == ORACLE_GRAD_BF16 ? bf16_to_f32(((const uint16_t *)grad)[k])
                                                        : ((const float *)grad)[k];

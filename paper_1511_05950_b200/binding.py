@@ -39,7 +39,7 @@ LOG_DTYPE = np.dtype([
 
 EXPORTS = (
     "ps_create", "ps_destroy", "ps_bind_state", "ps_init_weights", "ps_bind_staging",
-    "ps_set_option", "ps_get_option", "ps_pull_weights", "ps_pull_weights_host", "ps_pull_weights_host_async",
+    "ps_set_option", "ps_get_option", "ps_set_alpha0", "ps_pull_weights", "ps_pull_weights_host", "ps_pull_weights_host_async",
     "ps_push_gradient", "ps_push_gradient_host", "ps_apply_update", "ps_flush", "ps_synchronize",
     "ps_get_update_log", "ps_peek_state", "ps_kernel_time", "ps_last_cuda_error", "ps_status_string",
 )
@@ -67,6 +67,7 @@ def _load() -> C.CDLL:
         "ps_bind_staging": [vp, vp, i64, i32],
         "ps_set_option": [vp, i32, i64],
         "ps_get_option": [vp, i32, C.POINTER(i64)],
+        "ps_set_alpha0": [vp, f32],
         "ps_pull_weights": [vp, vp, C.POINTER(i64)],
         "ps_pull_weights_host": [vp, vp, C.POINTER(i64)],
         "ps_pull_weights_host_async": [vp, vp, C.POINTER(i64)],
@@ -99,6 +100,7 @@ ps_init_weights = lib.ps_init_weights
 ps_bind_staging = lib.ps_bind_staging
 ps_set_option = lib.ps_set_option
 ps_get_option = lib.ps_get_option
+ps_set_alpha0 = lib.ps_set_alpha0
 ps_pull_weights = lib.ps_pull_weights
 ps_pull_weights_host = lib.ps_pull_weights_host
 ps_pull_weights_host_async = lib.ps_pull_weights_host_async
@@ -200,6 +202,10 @@ class ParameterServer:
 
     def set_option(self, key: int, value: int) -> None:
         _check(ps_set_option(self._h, key, int(value)), "ps_set_option")
+
+    def set_alpha0(self, alpha0: float) -> None:
+        """Base learning rate for gradients pushed from now on."""
+        _check(ps_set_alpha0(self._h, alpha0), "ps_set_alpha0")
 
     def get_option(self, key: int) -> int:
         out = C.c_int64()

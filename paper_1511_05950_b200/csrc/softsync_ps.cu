@@ -22,6 +22,7 @@ using softsync::LaunchParams;
 struct Entry {                 // one pushed gradient waiting for its update
     int32_t learner;
     int64_t push_index, ts_grad, tau, sigma;
+    float alpha0;              // base rate in force when the gradient arrived
     const void *grad;
     int slot;                  // staging slot it occupies, -1 if borrowed from the caller
 };
@@ -156,7 +157,6 @@ void build_launch(ps_ctx *ps, int T, LaunchParams<MAXE> &p, std::vector<ps_log_e
     p.w = ps->w; p.v = ps->v; p.n = ps->n;
     p.momentum = ps->momentum; p.T = T; p.c = ps->c;
     vector_ok = aligned16(ps->w) && aligned16(ps->v);
-    const double alpha0 = static_cast<double>(ps->alpha0);
     const double wd = static_cast<double>(ps->weight_decay);
     for (int t = 0; t < T; ++t) {
         std::vector<Entry> &grp = ps->ready[t];
@@ -164,7 +164,8 @@ void build_launch(ps_ctx *ps, int T, LaunchParams<MAXE> &p, std::vector<ps_log_e
         double sum = 0.0;
         for (int l = 0; l < ps->c; ++l) {
             const Entry &en = grp[l];
-            const float s = static_cast<float>(alpha0 / (static_cast<double>(ps->c) * static_cast<double>(en.sigma)));
+            const float s = static_cast<float>(static_cast<double>(en.alpha0) /
+                                               (static_cast<double>(ps->c) * static_cast<double>(en.sigma)));
             p.s[t * ps->c + l] = s;
             p.g[t * ps->c + l] = en.grad;
             vector_ok = vector_ok && aligned16(en.grad);
@@ -264,6 +265,7 @@ int push_common(ps_ctx *ps, int learner, const void *grad_dev, int64_t ts, int s
     en.ts_grad = ts;
     en.tau = i - ts;                                      // staleness (Section 2.1)
     en.sigma = ps->modulation == PS_MOD_INV_STALENESS ? std::max<int64_t>(en.tau, 1) : 1;
+    en.alpha0 = ps->alpha0;
     en.grad = grad_dev;
     en.slot = slot;
     ps->push_count[learner] += 1;
@@ -441,6 +443,13 @@ int ps_get_option(ps_t *ps, int key, int64_t *value)
     case PS_OPT_BLOCK_THREADS: *value = ps->block_threads; return PS_OK;
     default: return PS_ERR_INVALID_ARG;
     }
+}
+
+int ps_set_alpha0(ps_t *ps, float alpha0)
+{
+    if (!is_live(ps) || !(alpha0 == alpha0)) return PS_ERR_INVALID_ARG;
+    ps->alpha0 = alpha0;
+    return PS_OK;
 }
 
 int ps_apply_update(ps_t *ps)

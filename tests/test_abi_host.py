@@ -101,6 +101,18 @@ def test_schedule_matches_reference_bit_exactly(model, lam, n, mod, fuse_t, lazy
     assert P.ps_destroy(h) == 0
 
 
+def test_rate_schedule_applies_to_later_pushes_only():
+    rc, h = make(2, 1, alpha0=0.5, m=0.0, wd=0.0)
+    assert P.ps_push_gradient(h, 0, FAKE_GRAD, 0) == P.PS_OK
+    assert P.ps_set_alpha0(h, 0.25) == 0
+    assert P.ps_set_alpha0(h, float("nan")) == P.PS_ERR_INVALID_ARG
+    assert P.ps_push_gradient(h, 1, FAKE_GRAD, 0) == P.PS_READY
+    assert P.ps_apply_update(h) == 1
+    ts, log = fetch_log(h, 2)
+    assert log["scale"].tolist() == [0.25, 0.125]          # as in the hand-worked example
+    P.ps_destroy(h)
+
+
 def test_logical_clock_runs_ahead_of_applied_clock():
     rc, h = make(2, 2)
     ts, a, l = C.c_int64(), C.c_int64(), C.c_int64()

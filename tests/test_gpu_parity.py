@@ -145,6 +145,46 @@ def test_sweep_point_with_uniform_staleness(c, grad_dtype):
     assert log["sigma"].max() > 1 or c == 1
 
 
+def test_rate_schedule_matches_reference():
+    """alpha0 lowered in steps while gradients are in flight (Section 4.3): a gradient keeps the rate
+    that was in force when it was pushed, also across fused passes."""
+    from tests.gpu_harness import as_reference_grad
+    dev = torch.device("cuda", 0)
+    n_el, lam, n = 50003, 6, 2
+    kinds, learners = R.simulate_arrivals("lognormal", lam, 90, 6)
+    w0 = G.initial_weights(layouts.flat(n_el), 6)
+    ps = P.ParameterServer(n_el, lam, n, 0.04, 0.9, 5e-4, fuse_t=4, device=dev)
+    ps.init_weights(w0.to(dev))
+    refs = {prec: R.ReferencePS(n_el, lam, n, 0.04, 0.9, 5e-4, R.MOD_INV_STALENESS, prec) for prec in (32, 64)}
+    for r in refs.values():
+        r.set_weights(w0.numpy())
+    pulled, counts, pushes, rate = {}, {}, 0, 0.04
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == 0:
+            pulled[l] = ps.pull_weights()
+            for r in refs.values():
+                assert r.pull(l) == pulled[l]
+            continue
+        if pushes % 11 == 5:
+            rate = rate * 0.5
+            ps.set_alpha0(rate)
+            for r in refs.values():
+                r.set_alpha0(rate)
+        b = counts.get(l, 0); counts[l] = b + 1
+        g = G.gradient(6, l, b, n_el, 1e-3, device=dev)
+        for r in refs.values():
+            r.push(l, as_reference_grad(g))
+        ps.push_gradient(l, g, pulled[l])
+        pushes += 1
+        if ps.timestamps()[1] - ps.timestamps()[0] >= 4:
+            ps.apply_update()
+    ps.flush(); ps.synchronize()
+    w, v, log = ps.w.cpu().numpy(), ps.v.cpu().numpy(), ps.update_log()
+    ps.destroy()
+    assert_parity(w, v, log, {prec: (*r.state(), r.log()) for prec, r in refs.items()}, TOL_FP32)
+    assert len(np.unique(log["scale"] * log["sigma"])) > 3
+
+
 def test_zero_parameters():
     _simple(0, 4, 2, 12)
 

@@ -25,7 +25,8 @@ MUTANTS = {
     "no_averaging": ("update_rule.inc", "((double)c * (double)sigma[l])", "((double)sigma[l])"),
     "wrong_gradient_index": ("update_rule.inc", "acc = acc + s[l] * grads[l][k];", "acc = acc + s[l] * grads[0][k];"),
     "wrong_scale_index": ("update_rule.inc", "acc = acc + s[l] * grads[l][k];", "acc = acc + s[0] * grads[l][k];"),
-    "decay_unmodulated": ("update_rule.inc", "const REAL d = ROUND_SCALE(wd * S);", "const REAL d = ROUND_SCALE(wd * alpha0);"),
+    "decay_unmodulated": ("update_rule.inc", "const REAL d = ROUND_SCALE(wd * S);", "const REAL d = ROUND_SCALE(wd * alpha0[0]);"),
+    "rate_at_apply_time": ("softsync_oracle.c", "alpha0[l] = ps->pending[order[l]].alpha0;", "alpha0[l] = ps->alpha0;"),
     "staleness_plus_one": ("softsync_oracle.c", "sigma = tau > 0 ? tau : 1;", "sigma = tau + 1;"),
     "staleness_ignored": ("softsync_oracle.c", "sigma = tau > 0 ? tau : 1;", "sigma = 1;"),
     "clock_jumps": ("softsync_oracle.c", "ps->ts += 1;", "ps->ts += ps->c;"),
@@ -44,6 +45,8 @@ def _pins():
         TU.test_single_learner_matches_library_sgd_optimizer,
         lambda: TU.test_one_softsync_with_barrier_is_synchronous_averaged_sgd(4),
         TU.test_downpour_case_is_per_push_sgd,
+        TU.test_step_schedule_without_momentum_is_library_sgd_with_a_changing_rate,
+        TU.test_rate_in_force_at_arrival_enters_the_geometric_sum,
         lambda: TU.test_plain_rule_is_a_weighted_sum_of_gradients("exp", 12, 3),
         TU.test_momentum_is_a_geometric_sum_of_past_steps,
         TU.test_decay_and_momentum_follow_the_linear_recurrence_in_matrix_form,

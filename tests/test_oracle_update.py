@@ -36,6 +36,9 @@ def test_hand_worked_examples_exact(example, precision):
         if ev[0] == "pull":
             ps.pull(ev[1])
             continue
+        if ev[0] == "alpha0":
+            ps.set_alpha0(ev[1])
+            continue
         fired = ps.push(ev[1], np.asarray(ev[2], np.float32))
         if fired:
             exp = ex["updates"][done]
@@ -152,6 +155,62 @@ def test_downpour_case_is_per_push_sgd():
     replay_reference(ps, k, l, grad)
     assert ps.timestamp == pushes
     assert rel_l2(ps.state()[0], w0.astype(np.float64) - a0 * total) < 1e-13
+
+
+def test_step_schedule_without_momentum_is_library_sgd_with_a_changing_rate():
+    """Section 4.3 lowers alpha0 in steps.  With one learner and no momentum the method is SGD whose
+    learning rate follows the schedule (library optimiser + StepLR)."""
+    n, steps = 32, 30
+    w0 = G.normal_like(G.stream_key(12, G.STREAM_WEIGHTS), 0, n, 0.01)
+    f32 = lambda x: float(np.float32(x))
+    lr0, wd = f32(0.1), f32(5e-4)
+    ps = R.ReferencePS(n, 1, 1, lr0, 0.0, wd, R.MOD_INV_STALENESS, 64)
+    ps.set_weights(w0.numpy())
+    p = torch.nn.Parameter(w0.double().clone())
+    opt = torch.optim.SGD([p], lr=lr0, momentum=0.0, weight_decay=wd)
+    sched = torch.optim.lr_scheduler.StepLR(opt, step_size=10, gamma=0.5)     # exact in binary
+    for s in range(steps):
+        ps.set_alpha0(opt.param_groups[0]["lr"])
+        g = G.gradient(12, 0, s, n, 1e-2)
+        ps.pull(0)
+        ps.push(0, g.numpy())
+        p.grad = g.double()
+        opt.step()
+        sched.step()
+    assert opt.param_groups[0]["lr"] == lr0 / 8
+    assert rel_l2(ps.state()[0], p.detach().numpy()) < 1e-13
+
+
+def test_rate_in_force_at_arrival_enters_the_geometric_sum():
+    """With momentum the step of update i is u_i = sum_l alpha0(at arrival of l)/(c sigma_l) g_l and
+    v_K = sum_i m^(K-1-i) u_i, whatever alpha0 is later."""
+    lam, n, n_el, pushes = 4, 2, 8, 40
+    c = lam // n
+    m = float(np.float32(0.5))
+    k, l = R.simulate_arrivals("exp", lam, pushes, 3)
+    tau, _ = staleness_by_recount(k, l, c)
+    ps = R.ReferencePS(n_el, lam, n, 0.25, m, 0.0, R.MOD_INV_STALENESS, 64)
+    ps.set_weights(np.zeros(n_el, np.float32))
+    seen, rates, counts = [], [], {}
+    rate = 0.25
+    for kind, who in zip(k.tolist(), l.tolist()):
+        if kind == 0:
+            ps.pull(who)
+            continue
+        if len(seen) % 7 == 3:
+            rate = rate / 2
+            ps.set_alpha0(rate)
+        b = counts.get(who, 0); counts[who] = b + 1
+        g = G.gradient(13, who, b, n_el, 1e-2).numpy()
+        seen.append(g.astype(np.float64)); rates.append(rate)
+        ps.push(who, g)
+    K = pushes // c
+    scaled = (np.asarray(rates[:K * c]) / (c * np.maximum(tau[:K * c], 1)))[:, None] * np.stack(seen[:K * c])
+    u = scaled.reshape(K, c, n_el).sum(1)
+    i = np.arange(K)
+    w, v = ps.state()
+    assert rel_l2(v, ((m ** (K - 1 - i))[:, None] * u).sum(0)) < 1e-12
+    assert rel_l2(w, -(((1 - m ** (K - i)) / (1 - m))[:, None] * u).sum(0)) < 1e-12
 
 
 # ---------------------------------------------------------------- closed forms

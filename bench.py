@@ -172,6 +172,9 @@ def run_ours(args, cfg, rank, world, local_rank):
     ps = P.ParameterServer(n, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
                            cfg.modulation, cfg.grad_dtype, fuse_t, device=dev)
     ps.init_weights(G.initial_weights(layout, cfg.seed + rank, cfg.weight_std, device=dev))
+    # every gradient buffer exists before the first update, so consecutive update kernels may overlap
+    # their launch ramps (the option's contract)
+    ps.set_option(P.PS_OPT_OVERLAP_LAUNCH, 0 if args.no_overlap else 1)
     pool_n = max(POOL_BUFFERS, 2 * cfg.c * fuse_t)
     pool = [G.gradient(cfg.seed + rank, i, 0, n, cfg.grad_std, dtype=tdt, device=dev) for i in range(pool_n)]
     total_steps = args.warmup + args.steps
@@ -264,6 +267,7 @@ def run_ours(args, cfg, rank, world, local_rank):
             "num_params": n, "lambda": cfg.num_learners, "n": cfg.n, "c": cfg.c, "fuse_t": fuse_t,
             "grad_dtype": cfg.grad_dtype, "arrivals": cfg.arrival_model, "alpha0": cfg.alpha0,
             "momentum": cfg.momentum, "weight_decay": cfg.weight_decay, "modulation": cfg.modulation,
+            "launch": "ordinary" if args.no_overlap else "programmatic dependent launch (PS_OPT_OVERLAP_LAUNCH=1)",
             "parallelism": "replicas only (independent servers, no data-path collective)" if world > 1 else "1 GPU",
             "l2": "inputs larger than L2: each step streams %.2f GB from %d rotating gradient buffers"
                   % (abytes / 1e9, pool_n),
@@ -422,6 +426,7 @@ def main():
     ap.add_argument("--workload", default="large_softsync", choices=sorted(configs.BY_NAME))
     ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true", help="ordinary launches instead of programmatic dependent ones")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
     ap.add_argument("--num-params", type=int, default=0,
                     help="run the workload's protocol on a flat vector of this many parameters (profiler captures)")

@@ -59,8 +59,15 @@ enum ps_option {
     PS_OPT_LOG_UPDATES = 5,               /* how many most recent updates the log keeps (default 65536) */
     PS_OPT_TIMING = 6,                    /* 1: bracket every update kernel with CUDA events (ps_kernel_time) */
     PS_OPT_KERNEL = 7,                    /* ps_kernel_choice (default PS_KERNEL_AUTO) */
+    PS_OPT_OVERLAP_LAUNCH = 9,            /* 1: update kernels are launched as programmatic dependents (see below); default 0 */
     PS_OPT_BLOCK_THREADS = 8              /* threads per block: 128, 256 or 512; 0 = default (128) */
 };
+
+/* PS_OPT_OVERLAP_LAUNCH = 1 lets an update kernel start while the previous kernel on the stream is still
+ * draining: it fetches its gradients at once and waits for the previous kernel only before it reads
+ * theta and v.  The caller promises in return that no gradient buffer is produced by the kernel that
+ * directly precedes a ps_apply_update on the server's stream (gradients written by earlier kernels, by
+ * copies, or on other streams with proper ordering are fine).  Results are bit-identical either way. */
 
 enum ps_kernel_choice {
     PS_KERNEL_AUTO = 0,                   /* vector kernel when every pointer is 16-byte aligned, else scalar */

@@ -49,7 +49,7 @@ struct ps_ctx {
     cudaStream_t stream = nullptr;
     int64_t queue_groups = 64;
     int64_t log_updates = 65536;
-    int timing = 0, kernel_choice = PS_KERNEL_AUTO, block_threads = 0;
+    int timing = 0, kernel_choice = PS_KERNEL_AUTO, block_threads = 0, overlap_launch = 0;
     int sm_count = 0;
 
     int64_t ts_applied = 0;                // updates whose kernel has been enqueued
@@ -108,8 +108,16 @@ constexpr int kHeadBf16 = 8;         // same for bf16 gradients
 template <typename GT, int VEC, int EC, bool MORE, int MAXE>
 cudaError_t launch_variant(const LaunchParams<MAXE> &p, int blocks, int threads, cudaStream_t stream)
 {
-    softsync::softsync_update_kernel<GT, VEC, EC, MORE, kChunk, MAXE><<<blocks, threads, 0, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+    cfg.blockDim = dim3(static_cast<unsigned>(threads));
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, softsync::softsync_update_kernel<GT, VEC, EC, MORE, kChunk, MAXE>, p);
 }
 
 // E = T*c <= HEAD: the straight-line instantiation with exactly E loads up front.
@@ -156,6 +164,7 @@ void build_launch(ps_ctx *ps, int T, LaunchParams<MAXE> &p, std::vector<ps_log_e
 {
     p.w = ps->w; p.v = ps->v; p.n = ps->n;
     p.momentum = ps->momentum; p.T = T; p.c = ps->c;
+    p.overlap = ps->overlap_launch;
     vector_ok = aligned16(ps->w) && aligned16(ps->v);
     const double wd = static_cast<double>(ps->weight_decay);
     for (int t = 0; t < T; ++t) {
@@ -421,6 +430,9 @@ int ps_set_option(ps_t *ps, int key, int64_t value)
     case PS_OPT_KERNEL:
         if (value < PS_KERNEL_AUTO || value > PS_KERNEL_VECTOR) return PS_ERR_INVALID_ARG;
         ps->kernel_choice = static_cast<int>(value); return PS_OK;
+    case PS_OPT_OVERLAP_LAUNCH:
+        if (value != 0 && value != 1) return PS_ERR_INVALID_ARG;
+        ps->overlap_launch = static_cast<int>(value); return PS_OK;
     case PS_OPT_BLOCK_THREADS:
         if (value != 0 && value != 128 && value != 256 && value != 512) return PS_ERR_INVALID_ARG;
         ps->block_threads = static_cast<int>(value); return PS_OK;
@@ -441,6 +453,7 @@ int ps_get_option(ps_t *ps, int key, int64_t *value)
     case PS_OPT_TIMING: *value = ps->timing; return PS_OK;
     case PS_OPT_KERNEL: *value = ps->kernel_choice; return PS_OK;
     case PS_OPT_BLOCK_THREADS: *value = ps->block_threads; return PS_OK;
+    case PS_OPT_OVERLAP_LAUNCH: *value = ps->overlap_launch; return PS_OK;
     default: return PS_ERR_INVALID_ARG;
     }
 }

@@ -32,6 +32,7 @@ struct LaunchParams {
     float momentum;
     int T;                // groups in this pass
     int c;                // gradients per group
+    int overlap;          // 1: launched as a programmatic dependent; gradients may be fetched early
     float d[kMaxFuseT];
     float s[MAXE];
     const void *g[MAXE];
@@ -113,6 +114,12 @@ __device__ __forceinline__ void store_state(float *p, const float (&x)[VEC])
     }
 }
 
+// Programmatic dependent launch (sm_90+): a kernel launched with the stream-serialisation
+// attribute may start while the previous kernel on the stream is draining; it must not touch
+// that kernel's output before griddep_wait() returns.  Both are no-ops in an ordinary launch.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- running state of one fragment while its gradients stream through -------
 template <int VEC>
 struct Fragment {
@@ -162,6 +169,7 @@ __device__ __forceinline__ void update_fragment(const LaunchParams<MAXE> &p, lon
     Raw<GT, VEC> head[EC > 0 ? EC : 1];
 #pragma unroll
     for (int e = 0; e < EC; ++e) load_raw(head[e], p.g[e], i);
+    if (p.overlap) griddep_wait();                       // theta and v are the previous update's output
     load_state<VEC>(p.w + first, f.w);
     load_state<VEC>(p.v + first, f.v);
     f.l = 0; f.t = 0;
@@ -194,6 +202,7 @@ __global__ void softsync_update_kernel(const __grid_constant__ LaunchParams<MAXE
 {
     const long long nfrag = p.n / VEC;
     const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (p.overlap) griddep_launch_dependents();          // the next pass may start filling free SM slots
     if (tid < nfrag)
         update_fragment<GT, VEC, EC, MORE, K, MAXE>(p, tid, tid * VEC);
     if constexpr (VEC > 1) {

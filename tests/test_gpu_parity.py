@@ -185,6 +185,51 @@ def test_rate_schedule_matches_reference():
     assert len(np.unique(log["scale"] * log["sigma"])) > 3
 
 
+@pytest.mark.parametrize("grad_dtype,fuse_t", [("fp32", 1), ("bf16", 4)])
+def test_overlapped_launch_gives_the_same_bits(grad_dtype, fuse_t):
+    """Update kernels launched as programmatic dependents (each may start while the previous one drains)
+    produce exactly what ordinary launches produce.  All gradients exist before the first update."""
+    dev = torch.device("cuda", 0)
+    n_el, lam, n, pushes = 2_000_003, 4, 2, 48
+    tdt = torch.bfloat16 if grad_dtype == "bf16" else torch.float32
+    kinds, learners = R.simulate_arrivals("exp", lam, pushes, 12)
+    w0 = G.initial_weights(layouts.flat(n_el), 12)
+    grads = {}
+    counts = {}
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == 1:
+            b = counts.get(l, 0); counts[l] = b + 1
+            grads[(l, b)] = G.gradient(12, l, b, n_el, 1e-3, dtype=tdt, device=dev)
+    torch.cuda.synchronize()
+    results = []
+    for overlap in (0, 1):
+        ps = P.ParameterServer(n_el, lam, n, 0.01, 0.9, 5e-4, grad_dtype=grad_dtype, fuse_t=fuse_t, device=dev)
+        ps.set_option(P.PS_OPT_OVERLAP_LAUNCH, overlap)
+        assert ps.get_option(P.PS_OPT_OVERLAP_LAUNCH) == overlap
+        ps.init_weights(w0.to(dev))
+        torch.cuda.synchronize()
+        pulled, counts, ready = {}, {}, 0
+        for k, l in zip(kinds.tolist(), learners.tolist()):
+            if k == 0:
+                pulled[l] = ps.pull_weights()
+                continue
+            b = counts.get(l, 0); counts[l] = b + 1
+            ready += ps.push_gradient(l, grads[(l, b)], pulled[l])
+            if ready >= fuse_t:
+                ready -= ps.apply_update()
+        ps.flush(); ps.synchronize()
+        results.append((ps.w.cpu().numpy().copy(), ps.v.cpu().numpy().copy(), ps.update_log()))
+        ps.destroy()
+    assert np.array_equal(results[0][0], results[1][0]) and np.array_equal(results[0][1], results[1][1])
+    assert np.array_equal(results[0][2], results[1][2])
+    ref = R.ReferencePS(n_el, lam, n, 0.01, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    from tests.gpu_harness import as_reference_grad
+    from tests.helpers import replay_reference
+    replay_reference(ref, kinds, learners, lambda l, b: as_reference_grad(grads[(l, b)]))
+    assert np.array_equal(results[1][0], ref.state()[0].astype(np.float32))
+
+
 def test_zero_parameters():
     _simple(0, 4, 2, 12)
 

@@ -66,8 +66,9 @@ enum ps_option {
 /* PS_OPT_OVERLAP_LAUNCH = 1 lets an update kernel start while the previous kernel on the stream is still
  * draining: it fetches its gradients at once and waits for the previous kernel only before it reads
  * theta and v.  The caller promises in return that no gradient buffer is produced by the kernel that
- * directly precedes a ps_apply_update on the server's stream (gradients written by earlier kernels, by
- * copies, or on other streams with proper ordering are fine).  Results are bit-identical either way. */
+ * directly precedes a ps_apply_update on the server's stream and may still be running (gradients written
+ * by earlier kernels, by kernels the host has already synchronised with, by copies, or on other streams
+ * with proper ordering are fine).  Results are bit-identical either way. */
 
 enum ps_kernel_choice {
     PS_KERNEL_AUTO = 0,                   /* vector kernel when every pointer is 16-byte aligned, else scalar */

@@ -214,3 +214,23 @@ def test_compute_without_a_gpu_fails_loudly():
     assert rc == P.PS_ERR_CUDA and not h.value
     with pytest.raises(P.SoftsyncError):
         P.ParameterServer(1024, 2, 1, 0.1, allocate=False)
+
+
+def test_unbuilt_library_fails_loudly_but_build_module_imports(tmp_path):
+    """A checkout without the built .so: the build module is importable, anything else raises."""
+    import shutil
+    import subprocess
+    import sys
+    pkg = tmp_path / "paper_1511_05950_b200"
+    pkg.mkdir()
+    src = os.path.join(ROOT, "paper_1511_05950_b200")
+    for fn in os.listdir(src):
+        if fn.endswith(".py"):
+            shutil.copy(os.path.join(src, fn), pkg / fn)
+    code = ("from paper_1511_05950_b200 import build\n"
+            "assert build.is_stale()\n"
+            "import paper_1511_05950_b200 as P\n"
+            "try:\n    P.ParameterServer\nexcept RuntimeError as e:\n    assert 'not built' in str(e); print('loud')\n")
+    out = subprocess.run([sys.executable, "-c", code], cwd=tmp_path, capture_output=True, text=True,
+                         env={**os.environ, "PYTHONPATH": str(tmp_path)})
+    assert out.returncode == 0 and "loud" in out.stdout, out.stderr

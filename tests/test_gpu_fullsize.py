@@ -34,7 +34,7 @@ def sample_indices(layout, count, seed):
     return torch.tensor(sorted(idx), dtype=torch.int64)
 
 
-def run_full(cfg, lazy, num_pushes=None):
+def run_full(cfg, lazy, num_pushes=None, overlap=False):
     dev = torch.device("cuda", 0)
     layout = cfg.layout()
     n = layout.num_params
@@ -55,6 +55,8 @@ def run_full(cfg, lazy, num_pushes=None):
     ps = P.ParameterServer(n, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
                            cfg.modulation, cfg.grad_dtype, cfg.fuse_t, device=dev)
     ps.init_weights(G.initial_weights(layout, cfg.seed, cfg.weight_std, device=dev))
+    if overlap:
+        ps.set_option(P.PS_OPT_OVERLAP_LAUNCH, 1)
     assert torch.equal(ps.w[idx_dev].cpu(), w0_s)      # same generator bits on both devices
 
     pulled, counts, ready = {}, {}, 0
@@ -75,6 +77,8 @@ def run_full(cfg, lazy, num_pushes=None):
             r.push(l, host)
         ready += ps.push_gradient(l, g, pulled[l])
         if ready and (not lazy or ready >= cfg.fuse_t):
+            if overlap:
+                torch.cuda.synchronize()      # the gradient just generated is complete before the update starts
             ready -= ps.apply_update()
     ps.flush()
     ps.synchronize()
@@ -97,7 +101,7 @@ def run_full(cfg, lazy, num_pushes=None):
 
 def test_large_softsync_full_size():
     """Config 3: 60,965,224 elements, lambda=18, n=4 (c=4), fp32 gradients, 500 updates."""
-    log = run_full(configs.LARGE_SOFTSYNC, lazy=False)
+    log = run_full(configs.LARGE_SOFTSYNC, lazy=False, overlap=True)     # launch mode bench.py times
     assert log["update"][-1] == 499
     assert 3.0 < log["tau"][200:].mean() < 5.5          # <tau> close to n = 4 (Section 2.4)
 

@@ -53,6 +53,7 @@ struct ps_ctx {
     int sm_count = 0;
 
     int64_t ts_applied = 0;                // updates whose kernel has been enqueued
+    int64_t launches = 0;                  // update kernels enqueued so far
     std::deque<std::vector<Entry>> ready;  // complete groups, oldest first
     std::vector<Entry> filling;            // the group being collected (< c entries)
     std::vector<int64_t> push_count;       // per learner
@@ -165,6 +166,7 @@ void build_launch(ps_ctx *ps, int T, LaunchParams<MAXE> &p, std::vector<ps_log_e
     p.w = ps->w; p.v = ps->v; p.n = ps->n;
     p.momentum = ps->momentum; p.T = T; p.c = ps->c;
     p.overlap = ps->overlap_launch;
+    p.reverse = static_cast<int>(ps->launches & 1);      // zig-zag over the vector from launch to launch
     vector_ok = aligned16(ps->w) && aligned16(ps->v);
     const double wd = static_cast<double>(ps->weight_decay);
     for (int t = 0; t < T; ++t) {
@@ -239,6 +241,7 @@ int apply_groups(ps_ctx *ps, int T)
             ps->timed.push_back(tl);
         }
     }
+    ps->launches += 1;
     // the launch is enqueued: advance the clock, release slots, publish the log
     for (int t = 0; t < T; ++t) {
         for (const Entry &en : ps->ready.front())

@@ -33,6 +33,7 @@ struct LaunchParams {
     int T;                // groups in this pass
     int c;                // gradients per group
     int overlap;          // 1: launched as a programmatic dependent; gradients may be fetched early
+    int reverse;          // 1: blocks walk the vector from its end (alternates from launch to launch)
     float d[kMaxFuseT];
     float s[MAXE];
     const void *g[MAXE];
@@ -203,8 +204,12 @@ __global__ void softsync_update_kernel(const __grid_constant__ LaunchParams<MAXE
     const long long nfrag = p.n / VEC;
     const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (p.overlap) griddep_launch_dependents();          // the next pass may start filling free SM slots
-    if (tid < nfrag)
-        update_fragment<GT, VEC, EC, MORE, K, MAXE>(p, tid, tid * VEC);
+    if (tid < nfrag) {
+        // Successive launches walk the vector in opposite directions: the part of theta and v that the
+        // previous launch touched last is still in the L2 and is the first thing this launch needs.
+        const long long i = p.reverse ? nfrag - 1 - tid : tid;
+        update_fragment<GT, VEC, EC, MORE, K, MAXE>(p, i, i * VEC);
+    }
     if constexpr (VEC > 1) {
         const long long done = nfrag * VEC;
         if (tid < p.n - done)

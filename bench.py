@@ -175,6 +175,8 @@ def run_ours(args, cfg, rank, world, local_rank):
     # every gradient buffer exists before the first update, so consecutive update kernels may overlap
     # their launch ramps (the option's contract)
     ps.set_option(P.PS_OPT_OVERLAP_LAUNCH, 0 if args.no_overlap else 1)
+    if args.bf16_mirror:
+        ps.bind_weight_mirror()                    # every pass also writes theta as bf16 (2 more bytes per element)
     pool_n = max(POOL_BUFFERS, 2 * cfg.c * fuse_t)
     pool = [G.gradient(cfg.seed + rank, i, 0, n, cfg.grad_std, dtype=tdt, device=dev) for i in range(pool_n)]
     total_steps = args.warmup + args.steps
@@ -253,7 +255,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     elems_per_step = cfg.c * n * groups_per_step
     value = whole_job_value(world, elems_per_step, args.steps, elapsed_ms)
     e2e_value = whole_job_value(world, elems_per_step, e2e_steps, e2e_ms) if e2e_steps else None
-    abytes = algorithmic_bytes(n, cfg.c * fuse_t, gbytes)
+    abytes = algorithmic_bytes(n, cfg.c * fuse_t, gbytes) + (2 * n if args.bf16_mirror else 0)
     peak, peak_kind = hbm_peak()
     achieved = abytes / (kern_ms * 1e-3) / 1e9
     result = {
@@ -267,6 +269,7 @@ def run_ours(args, cfg, rank, world, local_rank):
             "num_params": n, "lambda": cfg.num_learners, "n": cfg.n, "c": cfg.c, "fuse_t": fuse_t,
             "grad_dtype": cfg.grad_dtype, "arrivals": cfg.arrival_model, "alpha0": cfg.alpha0,
             "momentum": cfg.momentum, "weight_decay": cfg.weight_decay, "modulation": cfg.modulation,
+            "bf16_mirror": bool(args.bf16_mirror),
             "launch": "ordinary" if args.no_overlap else "programmatic dependent launch (PS_OPT_OVERLAP_LAUNCH=1)",
             "parallelism": "replicas only (independent servers, no data-path collective)" if world > 1 else "1 GPU",
             "l2": "inputs larger than L2: each step streams %.2f GB from %d rotating gradient buffers"
@@ -279,7 +282,7 @@ def run_ours(args, cfg, rank, world, local_rank):
                 "h2d_bytes_per_step": cfg.c * fuse_t * n * gbytes, "d2h_bytes_per_step": n * 4,
                 "ms_per_step": e2e_ms / e2e_steps if e2e_steps else None},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": TRAFFIC.get(cfg.name), "of": peak_kind,
+                     "frac": achieved / peak, "traffic": None if args.bf16_mirror else TRAFFIC.get(cfg.name), "of": peak_kind,
                      "kernel_ms": kern_ms, "algorithmic_bytes": abytes,
                      "how": "CUDA events around the %d back-to-back launches of the timed region / %d "
                             "(inter-launch gaps included)" % (args.steps, args.steps)},
@@ -427,6 +430,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="ordinary launches instead of programmatic dependent ones")
+    ap.add_argument("--bf16-mirror", action="store_true",
+                    help="variant: keep a bf16 copy of the weights current in the same pass (+2 bytes per element)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
     ap.add_argument("--num-params", type=int, default=0,
                     help="run the workload's protocol on a flat vector of this many parameters (profiler captures)")

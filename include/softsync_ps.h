@@ -113,6 +113,14 @@ int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev);
  * momentum, resets the timestamp to 0 and drops pending gradients and the log. */
 int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host);
 
+/* Binds a caller-owned device buffer of num_params bf16 values (2-byte aligned; 16-byte aligned keeps the
+ * vector kernel) that from now on always holds theta rounded to nearest-even bf16: it is filled at once
+ * (and by ps_init_weights), and every ps_apply_update rewrites it in the same pass that updates theta
+ * (2 more bytes per element instead of a separate conversion pass).  Learners that compute in bf16 can
+ * read it in place after the update, or take a copy with ps_pull_weights_bf16.  NULL unbinds.
+ * Not in the paper (its weights are 4-byte, Section 4.1). */
+int ps_bind_weight_mirror(ps_t *ps, void *mirror_bf16_dev);
+
 /* Binds `num_slots` caller-owned device slots of `slot_bytes` each (a multiple of 16, at least
  * num_params * gradient size; base 16-byte aligned) that ps_push_gradient_host copies into. */
 int ps_bind_staging(ps_t *ps, void *slots_dev, int64_t slot_bytes, int num_slots);
@@ -130,6 +138,10 @@ int ps_set_alpha0(ps_t *ps, float alpha0);
  * theta_i (num_params fp32) is copied to out_dev on the stream, so the weights always belong to
  * the returned timestamp.  out_dev == NULL returns the timestamp only. */
 int ps_pull_weights(ps_t *ps, float *out_dev, int64_t *ts);
+
+/* pullWeights for bf16 learners: like ps_pull_weights with out_dev != NULL, but copies the bf16 mirror
+ * (num_params * 2 bytes).  Needs ps_bind_weight_mirror. */
+int ps_pull_weights_bf16(ps_t *ps, void *out_bf16_dev, int64_t *ts);
 
 /* Same, into host memory; returns after the copy has completed. */
 int ps_pull_weights_host(ps_t *ps, float *out_host, int64_t *ts);

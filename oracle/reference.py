@@ -47,6 +47,8 @@ def load(path: str) -> C.CDLL:
         L.oracle_ps_push.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int]
         L.oracle_ps_push_with_timestamp.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int64]
         L.oracle_ps_get_state.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_ps_get_weights_bf16.argtypes = [C.c_void_p, C.c_void_p]
+        L.oracle_round_to_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.oracle_ps_log_size.restype = C.c_int64
         L.oracle_ps_log_size.argtypes = [C.c_void_p]
         L.oracle_ps_get_log.argtypes = [C.c_void_p, C.c_void_p]
@@ -85,6 +87,14 @@ def simulate_arrivals(model: str, num_learners: int, num_pushes: int, seed: int)
     if n < 0:
         raise ValueError("oracle_simulate_arrivals rejected its arguments")
     return kind[:n].copy(), learner[:n].copy()
+
+
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """fp32 -> bf16 bit patterns (uint16), round to nearest even, by the reference's own routine."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.size, dtype=np.uint16)
+    lib().oracle_round_to_bf16(x.ctypes.data, out.ctypes.data, x.size)
+    return out.reshape(x.shape)
 
 
 class ReferencePS:
@@ -151,6 +161,13 @@ class ReferencePS:
         v = np.empty(self.num_params, dtype=np.float64)
         lib().oracle_ps_get_state(self._h, w.ctypes.data, v.ctypes.data)
         return w, v
+
+    def weights_bf16(self) -> np.ndarray:
+        """Weights rounded to bf16 (uint16 bit patterns); fp32 state only."""
+        out = np.empty(self.num_params, dtype=np.uint16)
+        if lib().oracle_ps_get_weights_bf16(self._h, out.ctypes.data) != 0:
+            raise ValueError("bf16 weights are defined for precision 32 only")
+        return out
 
     def log(self) -> np.ndarray:
         n = lib().oracle_ps_log_size(self._h)

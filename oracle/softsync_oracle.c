@@ -252,6 +252,31 @@ void oracle_ps_get_state(const oracle_ps *ps, double *w_out, double *v_out)
     }
 }
 
+/* fp32 -> bf16, round to nearest, ties to even: bf16 keeps the upper 16 bits of the fp32 pattern, so add
+ * half of the dropped part (0x7FFF plus the lowest kept bit) and truncate.  NaN maps to 0x7FFF. */
+static uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u; memcpy(&u, &f, sizeof u);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return 0x7FFF;
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+/* The weights as a bf16 learner would pull them (an extension: the paper's weights are 4-byte).
+ * Defined for the fp32 server state only. */
+int oracle_ps_get_weights_bf16(const oracle_ps *ps, uint16_t *out)
+{
+    if (ps->precision != 32) return -1;
+    for (int64_t k = 0; k < ps->N; ++k) out[k] = f32_to_bf16_rne(((const float *)ps->w)[k]);
+    return 0;
+}
+
+/* The same rounding on caller-supplied values (so that it can be pinned on its own). */
+void oracle_round_to_bf16(const float *in, uint16_t *out, int64_t n)
+{
+    for (int64_t k = 0; k < n; ++k) out[k] = f32_to_bf16_rne(in[k]);
+}
+
 int64_t oracle_ps_log_size(const oracle_ps *ps) { return ps->log_size; }
 
 void oracle_ps_get_log(const oracle_ps *ps, oracle_log_entry *out)

@@ -38,7 +38,8 @@ LOG_DTYPE = np.dtype([
 ], align=True)
 
 EXPORTS = (
-    "ps_create", "ps_destroy", "ps_bind_state", "ps_init_weights", "ps_bind_staging",
+    "ps_create", "ps_destroy", "ps_bind_state", "ps_init_weights", "ps_bind_staging", "ps_bind_weight_mirror",
+    "ps_pull_weights_bf16",
     "ps_set_option", "ps_get_option", "ps_set_alpha0", "ps_pull_weights", "ps_pull_weights_host", "ps_pull_weights_host_async",
     "ps_push_gradient", "ps_push_gradient_host", "ps_apply_update", "ps_flush", "ps_synchronize",
     "ps_get_update_log", "ps_peek_state", "ps_kernel_time", "ps_last_cuda_error", "ps_status_string",
@@ -65,6 +66,8 @@ def _load() -> C.CDLL:
         "ps_bind_state": [vp, vp, vp],
         "ps_init_weights": [vp, vp, i32],
         "ps_bind_staging": [vp, vp, i64, i32],
+        "ps_bind_weight_mirror": [vp, vp],
+        "ps_pull_weights_bf16": [vp, vp, C.POINTER(i64)],
         "ps_set_option": [vp, i32, i64],
         "ps_get_option": [vp, i32, C.POINTER(i64)],
         "ps_set_alpha0": [vp, f32],
@@ -98,6 +101,8 @@ ps_destroy = lib.ps_destroy
 ps_bind_state = lib.ps_bind_state
 ps_init_weights = lib.ps_init_weights
 ps_bind_staging = lib.ps_bind_staging
+ps_bind_weight_mirror = lib.ps_bind_weight_mirror
+ps_pull_weights_bf16 = lib.ps_pull_weights_bf16
 ps_set_option = lib.ps_set_option
 ps_get_option = lib.ps_get_option
 ps_set_alpha0 = lib.ps_set_alpha0
@@ -148,7 +153,7 @@ class ParameterServer:
         self._held = collections.deque()
         self._host_held = []          # pinned host gradients whose upload may still be in flight
         self._staging = None
-        self.w = self.v = None
+        self.w = self.v = self.mirror = None
         if device is None and (allocate or state is not None) and num_params > 0:
             device = torch.device("cuda", torch.cuda.current_device())
         self.device = device
@@ -200,6 +205,15 @@ class ParameterServer:
         _check(ps_bind_staging(self._h, buf.data_ptr(), slot_bytes, num_slots), "ps_bind_staging")
         self._staging = buf
 
+    def bind_weight_mirror(self, mirror: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Keep a bf16 copy of the weights current in `mirror` (allocated here if not given)."""
+        if mirror is None:
+            mirror = torch.empty(max(1, self.num_params), dtype=torch.bfloat16, device=self.device)
+        assert mirror.dtype == torch.bfloat16 and mirror.numel() >= self.num_params
+        _check(ps_bind_weight_mirror(self._h, mirror.data_ptr()), "ps_bind_weight_mirror")
+        self.mirror = mirror
+        return mirror
+
     def set_option(self, key: int, value: int) -> None:
         _check(ps_set_option(self._h, key, int(value)), "ps_set_option")
 
@@ -217,6 +231,11 @@ class ParameterServer:
         """Timestamp a gradient computed from now on must carry; fills `out` with the weights if given.
         non_blocking (host `out` only): return once the copy is enqueued; call synchronize() before reading."""
         ts = C.c_int64()
+        if out is not None and out.dtype == torch.bfloat16:
+            assert out.is_cuda and out.is_contiguous()
+            _check(ps_pull_weights_bf16(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_bf16")
+            self._held.clear()
+            return ts.value
         if out is not None and not out.is_cuda:
             assert out.dtype == torch.float32 and out.is_contiguous()
             if non_blocking:

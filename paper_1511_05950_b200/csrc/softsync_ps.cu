@@ -39,6 +39,7 @@ struct ps_ctx {
     int device = 0;
 
     float *w = nullptr, *v = nullptr;
+    unsigned short *mirror = nullptr;      // optional caller-owned bf16 copy of theta
     char *staging = nullptr;
     int64_t slot_bytes = 0;
     std::vector<int> free_slots;
@@ -167,7 +168,8 @@ void build_launch(ps_ctx *ps, int T, LaunchParams<MAXE> &p, std::vector<ps_log_e
     p.momentum = ps->momentum; p.T = T; p.c = ps->c;
     p.overlap = ps->overlap_launch;
     p.reverse = static_cast<int>(ps->launches & 1);      // zig-zag over the vector from launch to launch
-    vector_ok = aligned16(ps->w) && aligned16(ps->v);
+    p.mirror = ps->mirror;
+    vector_ok = aligned16(ps->w) && aligned16(ps->v) && aligned16(ps->mirror);
     const double wd = static_cast<double>(ps->weight_decay);
     for (int t = 0; t < T; ++t) {
         std::vector<Entry> &grp = ps->ready[t];
@@ -203,6 +205,18 @@ int order_after_readback(ps_ctx *ps)
         PS_CUDA(ps, cudaStreamWaitEvent(ps->stream, ps->weights_copied, 0));
         ps->copy_in_flight = false;
     }
+    return PS_OK;
+}
+
+// Rewrites the whole bf16 mirror from theta (set-up paths; updates keep it current themselves).
+int refresh_mirror(ps_ctx *ps)
+{
+    if (!ps->mirror || !ps->w || ps->n == 0) return PS_OK;
+    const int threads = 256;
+    const long long want = (ps->n + threads - 1) / threads;
+    const int blocks = static_cast<int>(std::min<long long>(want, static_cast<long long>(ps->sm_count) * 32));
+    softsync::mirror_kernel<<<blocks, threads, 0, ps->stream>>>(ps->w, ps->mirror, ps->n);
+    PS_CUDA(ps, cudaGetLastError());
     return PS_OK;
 }
 
@@ -382,6 +396,8 @@ int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host)
         if (rb != PS_OK) return rb;
         PS_CUDA(ps, cudaMemcpyAsync(ps->w, w_src, bytes, src_is_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, ps->stream));
         PS_CUDA(ps, cudaMemsetAsync(ps->v, 0, bytes, ps->stream));
+        const int rm = refresh_mirror(ps);
+        if (rm != PS_OK) return rm;
         if (src_is_host) PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
     }
     for (auto &grp : ps->ready) for (const Entry &en : grp) if (en.slot >= 0) ps->free_slots.push_back(en.slot);
@@ -391,6 +407,16 @@ int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host)
     ps->ts_applied = 0;
     ps->log.clear(); ps->log_first_update = 0;
     return PS_OK;
+}
+
+int ps_bind_weight_mirror(ps_t *ps, void *mirror_dev)
+{
+    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(mirror_dev) & 1u) return PS_ERR_INVALID_ARG;
+    if (mirror_dev && (mirror_dev == ps->w || mirror_dev == ps->v)) return PS_ERR_INVALID_ARG;
+    if (!ps->ready.empty()) return PS_ERR_INVALID_ARG;               // apply or flush first
+    ps->mirror = static_cast<unsigned short *>(mirror_dev);
+    return refresh_mirror(ps);
 }
 
 int ps_bind_staging(ps_t *ps, void *slots_dev, int64_t slot_bytes, int num_slots)
@@ -496,6 +522,18 @@ int ps_pull_weights(ps_t *ps, float *out_dev, int64_t *ts)
         if (ps->n) PS_CUDA(ps, cudaMemcpyAsync(out_dev, ps->w, static_cast<size_t>(ps->n) * sizeof(float),
                                                cudaMemcpyDeviceToDevice, ps->stream));
     }
+    *ts = ts_logical(ps);
+    return PS_OK;
+}
+
+int ps_pull_weights_bf16(ps_t *ps, void *out_dev, int64_t *ts)
+{
+    if (!is_live(ps) || !ts || !out_dev) return PS_ERR_INVALID_ARG;
+    if (!ps->mirror || (ps->n > 0 && (!ps->w || !ps->v))) return PS_ERR_NO_STATE;
+    const int r = ps_flush(ps);
+    if (r < 0) return r;
+    if (ps->n) PS_CUDA(ps, cudaMemcpyAsync(out_dev, ps->mirror, static_cast<size_t>(ps->n) * 2,
+                                           cudaMemcpyDeviceToDevice, ps->stream));
     *ts = ts_logical(ps);
     return PS_OK;
 }

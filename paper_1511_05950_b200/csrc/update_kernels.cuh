@@ -14,6 +14,7 @@
 // never contracted into an FMA).
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -34,6 +35,7 @@ struct LaunchParams {
     int c;                // gradients per group
     int overlap;          // 1: launched as a programmatic dependent; gradients may be fetched early
     int reverse;          // 1: blocks walk the vector from its end (alternates from launch to launch)
+    unsigned short *mirror;   // optional bf16 copy of theta, rewritten by every pass (nullptr: none)
     float d[kMaxFuseT];
     float s[MAXE];
     const void *g[MAXE];
@@ -121,6 +123,33 @@ __device__ __forceinline__ void store_state(float *p, const float (&x)[VEC])
 __device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// ---- bf16 mirror of theta: round to nearest even, stored as raw 16-bit patterns ----
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);       // .x = lo (low half), .y = hi
+    return *reinterpret_cast<const unsigned *>(&b);
+}
+template <int VEC>
+__device__ __forceinline__ void store_mirror(unsigned short *p, const float (&x)[VEC])
+{
+    if constexpr (VEC == 1) {
+        *p = __bfloat16_as_ushort(__float2bfloat16_rn(x[0]));
+    } else if constexpr (VEC == 4) {
+        __stcs(reinterpret_cast<uint2 *>(p), make_uint2(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3])));
+    } else {
+        __stcs(reinterpret_cast<uint4 *>(p), make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]),
+                                                         pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7])));
+    }
+}
+
+// theta -> bf16 mirror on its own (after ps_init_weights or when a mirror is bound).
+__global__ void mirror_kernel(const float *w, unsigned short *mirror, long long n)
+{
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += stride)
+        mirror[i] = __bfloat16_as_ushort(__float2bfloat16_rn(w[i]));
+}
+
 // ---- running state of one fragment while its gradients stream through -------
 template <int VEC>
 struct Fragment {
@@ -190,6 +219,7 @@ __device__ __forceinline__ void update_fragment(const LaunchParams<MAXE> &p, lon
     }
     store_state<VEC>(p.w + first, f.w);
     store_state<VEC>(p.v + first, f.v);
+    if (p.mirror) store_mirror<VEC>(p.mirror + first, f.w);
 }
 
 // One fragment of VEC elements per thread: the grid covers the vector exactly once

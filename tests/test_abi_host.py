@@ -201,6 +201,19 @@ def test_group_larger_than_one_launch_clamps_fusion():
     P.ps_destroy(h)
 
 
+def test_weight_mirror_argument_checks():
+    rc, h = make(2, 1)
+    assert P.ps_bind_weight_mirror(h, 0x1001) == P.PS_ERR_INVALID_ARG           # odd address
+    assert P.ps_bind_weight_mirror(None, 0x1000) == P.PS_ERR_INVALID_ARG
+    assert P.ps_bind_weight_mirror(h, 0x1000) == 0                              # zero parameters: nothing is written
+    ts = C.c_int64()
+    assert P.ps_pull_weights_bf16(h, None, C.byref(ts)) == P.PS_ERR_INVALID_ARG
+    assert P.ps_pull_weights_bf16(h, 0x2000, C.byref(ts)) == 0 and ts.value == 0
+    assert P.ps_bind_weight_mirror(h, None) == 0                                # unbind
+    assert P.ps_pull_weights_bf16(h, 0x2000, C.byref(ts)) == P.PS_ERR_NO_STATE
+    P.ps_destroy(h)
+
+
 def test_status_strings():
     assert P.status_string(P.PS_ERR_BAD_TIMESTAMP).startswith("gradient timestamp")
     assert P.status_string(0) == "ok"

@@ -230,6 +230,64 @@ def test_overlapped_launch_gives_the_same_bits(grad_dtype, fuse_t):
     assert np.array_equal(results[1][0], ref.state()[0].astype(np.float32))
 
 
+@pytest.mark.parametrize("grad_dtype,fuse_t,n_el,misalign", [
+    ("fp32", 1, 70003, 0), ("bf16", 4, 70005, 0), ("fp32", 3, 9999, 1), ("bf16", 1, 4097, 3), ("fp32", 1, 3, 0)])
+def test_bf16_weight_mirror_tracks_the_weights(grad_dtype, fuse_t, n_el, misalign):
+    """The bf16 copy written by the update pass equals the reference's weights rounded to bf16, bit for bit,
+    after set-up, after every update (fused or not, vector or scalar kernel) and through the bf16 pull."""
+    from tests.gpu_harness import as_reference_grad
+    dev = torch.device("cuda", 0)
+    tdt = torch.bfloat16 if grad_dtype == "bf16" else torch.float32
+    lam, n = 6, 3
+    kinds, learners = R.simulate_arrivals("exp", lam, 30, 8)
+    w0 = G.initial_weights(layouts.flat(n_el), 8)
+    ref = R.ReferencePS(n_el, lam, n, 0.05, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    ps = P.ParameterServer(n_el, lam, n, 0.05, 0.9, 5e-4, grad_dtype=grad_dtype, fuse_t=fuse_t, device=dev)
+    ps.init_weights(w0.to(dev))
+    guard = torch.full((n_el + misalign + 64,), 7.0, dtype=torch.bfloat16, device=dev)
+    mirror = ps.bind_weight_mirror(guard[misalign:misalign + n_el])
+
+    def bits(t):
+        return t.cpu().view(torch.int16).numpy().view(np.uint16)
+
+    assert np.array_equal(bits(mirror), ref.weights_bf16())               # filled when bound
+    pulled, counts, ready = {}, {}, 0
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == 0:
+            pulled[l] = ps.pull_weights()
+            ref.pull(l)
+            continue
+        b = counts.get(l, 0); counts[l] = b + 1
+        g = G.gradient(8, l, b, n_el, 1e-2, dtype=tdt, device=dev)
+        fired = ref.push(l, as_reference_grad(g))
+        ready += ps.push_gradient(l, g, pulled[l])
+        if ready >= fuse_t:
+            ready -= ps.apply_update()
+            if ready == 0:
+                assert np.array_equal(bits(mirror), ref.weights_bf16())
+    out = torch.empty(n_el, dtype=torch.bfloat16, device=dev)
+    assert ps.pull_weights(out) == ref.timestamp                              # flushes, then copies the mirror
+    assert np.array_equal(bits(out), ref.weights_bf16())
+    assert np.array_equal(ps.w[:n_el].cpu().numpy(), ref.state()[0].astype(np.float32))
+    assert (guard[:misalign] == 7.0).all() and (guard[misalign + n_el:] == 7.0).all()
+    ps.init_weights(w0.to(dev))                                               # re-initialising refreshes it
+    ref2 = R.round_to_bf16(w0.numpy())
+    assert np.array_equal(bits(mirror), ref2)
+    ps.destroy()
+
+
+def test_bf16_pull_needs_a_mirror():
+    dev = torch.device("cuda", 0)
+    ps = P.ParameterServer(64, 1, 1, 0.1, device=dev)
+    ps.init_weights(torch.zeros(64))
+    out = torch.empty(64, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(P.SoftsyncError) as e:
+        ps.pull_weights(out)
+    assert e.value.status == P.PS_ERR_NO_STATE
+    ps.destroy()
+
+
 def test_zero_parameters():
     _simple(0, 4, 2, 12)
 

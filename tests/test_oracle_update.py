@@ -334,6 +334,42 @@ def test_bf16_gradients_are_widened_exactly():
     assert a.timestamp == 15
 
 
+def test_bf16_rounding_matches_library_conversion_and_hand_cases():
+    """Round-to-nearest-even fp32 -> bf16: against torch's conversion on random and special values,
+    and against tie cases worked by hand (bf16 keeps 8 significand bits)."""
+    rng = np.random.default_rng(0)
+    bits = rng.integers(0, 1 << 32, size=200000, dtype=np.uint64).astype(np.uint32)
+    x = bits.view(np.float32)
+    x = x[np.isfinite(x)]
+    special = np.array([0.0, -0.0, np.inf, -np.inf, 1.0, -1.0, 3.3895314e38, 3.4028235e38, 1e-40, -1e-45,
+                        1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, 1.0 + 2.0 ** -9], np.float32)
+    x = np.concatenate([x, special])
+    got = R.round_to_bf16(x)
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(got, want)
+    # hand cases: 1 + 2^-8 is exactly half-way between 1 (0x3F80) and 1 + 2^-7 (0x3F81): ties go to the even 0x3F80;
+    # 1 + 3*2^-8 is half-way between 0x3F81 and 0x3F82: goes to the even 0x3F82; just above half-way goes up;
+    # the largest fp32 rounds to +inf (0x7F80).
+    hand = R.round_to_bf16(np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20,
+                                     1.0 + 2.0 ** -9, 3.4028235e38], np.float32))
+    assert hand.tolist() == [0x3F80, 0x3F82, 0x3F81, 0x3F80, 0x7F80]
+    assert R.round_to_bf16(np.array([np.nan], np.float32)).tolist() == [0x7FFF]
+
+
+def test_bf16_weights_are_the_rounded_fp32_state():
+    ps = R.ReferencePS(5, 1, 1, 0.5, 0.0, 0.0, R.MOD_INV_STALENESS, 32)
+    ps.set_weights(np.array([1.0, 2.0, 3.0, 4.0, 5.0], np.float32))
+    ps.pull(0)
+    ps.push(0, np.array([2.0 ** -8, 0.0, 3 * 2.0 ** -7, -1.0, 2.0 ** -6], np.float32) * -2)   # w += exact dyadics
+    w, _ = ps.state()
+    assert w.tolist() == [1.0 + 2.0 ** -8, 2.0, 3.0 + 3 * 2.0 ** -7, 3.0, 5.0 + 2.0 ** -6]
+    # 3 + 3*2^-7 = 1.5*(2 + 2^-6): the dropped bits are exactly half an ulp (2^-6 at this exponent) with an odd
+    # kept part: rounds up to 3 + 2^-5 (0x4042); 5 + 2^-6 is half-way between 5 (0x40A0) and 5 + 2^-5: stays even
+    assert ps.weights_bf16().tolist() == [0x3F80, 0x4000, 0x4042, 0x4040, 0x40A0]
+    with pytest.raises(ValueError):
+        R.ReferencePS(2, 1, 1, 0.1, 0.0, 0.0, R.MOD_INV_STALENESS, 64).weights_bf16()
+
+
 def test_fp32_reference_tracks_fp64_reference():
     """Noise floor of keeping the state in fp32, on the small benchmark shape."""
     from workloads import configs

@@ -104,8 +104,7 @@ bool entry_before(const Entry &a, const Entry &b)
 }
 
 constexpr int kChunk = 8;            // gradient loads in flight per thread beyond the first EC
-constexpr int kHeadFp32 = 16;        // largest compile-time first chunk, fp32 gradients
-constexpr int kHeadBf16 = 8;         // same for bf16 gradients
+constexpr int kHead = 16;            // largest compile-time first chunk of gradient loads
 
 template <typename GT, int VEC, int EC, bool MORE, int MAXE>
 cudaError_t launch_variant(const LaunchParams<MAXE> &p, int blocks, int threads, cudaStream_t stream)
@@ -137,7 +136,11 @@ cudaError_t launch_exact(int E, const LaunchParams<MAXE> &p, int blocks, int thr
 template <typename GT, int VEC, int HEAD, int MAXE>
 cudaError_t launch_vector(int E, const LaunchParams<MAXE> &p, int blocks, int threads, cudaStream_t stream)
 {
-    if (E <= HEAD) return launch_exact<GT, VEC, (HEAD < MAXE ? HEAD : MAXE), MAXE>(E, p, blocks, threads, stream);
+    if constexpr (MAXE <= HEAD) {                        // the small parameter block: T*c <= HEAD always
+        return launch_exact<GT, VEC, MAXE, MAXE>(E, p, blocks, threads, stream);
+    } else {
+        if (E <= HEAD) return cudaErrorInvalidValue;     // such launches use the small parameter block
+    }
     return launch_variant<GT, VEC, HEAD, true, MAXE>(p, blocks, threads, stream);   // HEAD loads, then chunks
 }
 
@@ -145,7 +148,7 @@ template <int MAXE>
 cudaError_t launch_update(ps_ctx *ps, const LaunchParams<MAXE> &p, bool vector_ok)
 {
     const bool bf16 = ps->grad_dtype == PS_GRAD_BF16;
-    const int vec = vector_ok ? (bf16 ? 8 : 4) : 1;
+    const int vec = vector_ok ? 4 : 1;
     const int threads = ps->block_threads ? ps->block_threads : 128;
     const long long frags = std::max<long long>(1, (p.n + vec - 1) / vec);
     const long long blocks = (frags + threads - 1) / threads;    // one fragment per thread
@@ -155,8 +158,8 @@ cudaError_t launch_update(ps_ctx *ps, const LaunchParams<MAXE> &p, bool vector_o
     if (!vector_ok)
         return bf16 ? launch_variant<GradBf16, 1, 0, true, MAXE>(p, b, threads, ps->stream)
                     : launch_variant<GradFp32, 1, 0, true, MAXE>(p, b, threads, ps->stream);
-    return bf16 ? launch_vector<GradBf16, 8, kHeadBf16, MAXE>(E, p, b, threads, ps->stream)
-                : launch_vector<GradFp32, 4, kHeadFp32, MAXE>(E, p, b, threads, ps->stream);
+    return bf16 ? launch_vector<GradBf16, 4, kHead, MAXE>(E, p, b, threads, ps->stream)
+                : launch_vector<GradFp32, 4, kHead, MAXE>(E, p, b, threads, ps->stream);
 }
 
 // Fills the scale table of one launch (Eq. 3 folded with the 1/c of Eq. 2) for the `T`

@@ -44,10 +44,10 @@ struct LaunchParams {
 struct GradFp32 {};
 struct GradBf16 {};
 
-// ---- raw 16-byte (or scalar) gradient fragments ---------------------------
+// ---- raw gradient fragments: 4 elements (16 bytes fp32, 8 bytes bf16) or one ----
 template <typename GT, int VEC> struct Raw;
 template <> struct Raw<GradFp32, 4> { float4 q; };
-template <> struct Raw<GradBf16, 8> { uint4 q; };
+template <> struct Raw<GradBf16, 4> { uint2 q; };
 template <> struct Raw<GradFp32, 1> { float q; };
 template <> struct Raw<GradBf16, 1> { unsigned short q; };
 
@@ -58,18 +58,17 @@ __device__ __forceinline__ float4 ld_stream_f4(const float4 *p)
                  : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(p));
     return r;
 }
-__device__ __forceinline__ uint4 ld_stream_u4(const uint4 *p)
+__device__ __forceinline__ uint2 ld_stream_u2(const uint2 *p)
 {
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    uint2 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
     return r;
 }
 
 __device__ __forceinline__ void load_raw(Raw<GradFp32, 4> &r, const void *base, long long i)
 { r.q = ld_stream_f4(reinterpret_cast<const float4 *>(base) + i); }
-__device__ __forceinline__ void load_raw(Raw<GradBf16, 8> &r, const void *base, long long i)
-{ r.q = ld_stream_u4(reinterpret_cast<const uint4 *>(base) + i); }
+__device__ __forceinline__ void load_raw(Raw<GradBf16, 4> &r, const void *base, long long i)
+{ r.q = ld_stream_u2(reinterpret_cast<const uint2 *>(base) + i); }
 __device__ __forceinline__ void load_raw(Raw<GradFp32, 1> &r, const void *base, long long i)
 { r.q = __ldg(reinterpret_cast<const float *>(base) + i); }
 __device__ __forceinline__ void load_raw(Raw<GradBf16, 1> &r, const void *base, long long i)
@@ -78,14 +77,10 @@ __device__ __forceinline__ void load_raw(Raw<GradBf16, 1> &r, const void *base, 
 // bf16 is the upper half of an fp32: widening is a shift, exact.
 __device__ __forceinline__ void widen(const Raw<GradFp32, 4> &r, float (&g)[4])
 { g[0] = r.q.x; g[1] = r.q.y; g[2] = r.q.z; g[3] = r.q.w; }
-__device__ __forceinline__ void widen(const Raw<GradBf16, 8> &r, float (&g)[8])
+__device__ __forceinline__ void widen(const Raw<GradBf16, 4> &r, float (&g)[4])
 {
-    const unsigned u[4] = {r.q.x, r.q.y, r.q.z, r.q.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        g[2 * j] = __uint_as_float(u[j] << 16);
-        g[2 * j + 1] = __uint_as_float(u[j] & 0xFFFF0000u);
-    }
+    g[0] = __uint_as_float(r.q.x << 16); g[1] = __uint_as_float(r.q.x & 0xFFFF0000u);
+    g[2] = __uint_as_float(r.q.y << 16); g[3] = __uint_as_float(r.q.y & 0xFFFF0000u);
 }
 __device__ __forceinline__ void widen(const Raw<GradFp32, 1> &r, float (&g)[1]) { g[0] = r.q; }
 __device__ __forceinline__ void widen(const Raw<GradBf16, 1> &r, float (&g)[1])
@@ -134,11 +129,9 @@ __device__ __forceinline__ void store_mirror(unsigned short *p, const float (&x)
 {
     if constexpr (VEC == 1) {
         *p = __bfloat16_as_ushort(__float2bfloat16_rn(x[0]));
-    } else if constexpr (VEC == 4) {
-        __stcs(reinterpret_cast<uint2 *>(p), make_uint2(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3])));
     } else {
-        __stcs(reinterpret_cast<uint4 *>(p), make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]),
-                                                         pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7])));
+        static_assert(VEC == 4, "fragments hold one or four elements");
+        __stcs(reinterpret_cast<uint2 *>(p), make_uint2(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3])));
     }
 }
 
@@ -191,7 +184,7 @@ __device__ __forceinline__ void consume(const LaunchParams<MAXE> &p, Fragment<VE
 // is consumed, so every thread has (EC + 2) independent 16-byte requests in
 // flight.  MORE = false: the launch has exactly EC entries and the code is
 // straight-line (no spare registers held for a loop that never runs).
-// MORE = true: entries beyond EC follow in chunks of K loads.
+// MORE = true: entries beyond EC follow in chunks of K loads, the last few one by one.
 template <typename GT, int VEC, int EC, bool MORE, int K, int MAXE>
 __device__ __forceinline__ void update_fragment(const LaunchParams<MAXE> &p, long long i, long long first)
 {
@@ -207,14 +200,18 @@ __device__ __forceinline__ void update_fragment(const LaunchParams<MAXE> &p, lon
     for (int e = 0; e < EC; ++e) consume<GT, VEC, MAXE>(p, f, head[e], e);
     if constexpr (MORE) {
         const int E = p.T * p.c;
-        for (int e0 = EC; e0 < E; e0 += K) {
+        int e0 = EC;
+        for (; e0 + K <= E; e0 += K) {                   // full chunks: K independent loads, no predicates
             Raw<GT, VEC> raw[K];
 #pragma unroll
-            for (int k = 0; k < K; ++k)
-                if (e0 + k < E) load_raw(raw[k], p.g[e0 + k], i);
+            for (int k = 0; k < K; ++k) load_raw(raw[k], p.g[e0 + k], i);
 #pragma unroll
-            for (int k = 0; k < K; ++k)
-                if (e0 + k < E) consume<GT, VEC, MAXE>(p, f, raw[k], e0 + k);
+            for (int k = 0; k < K; ++k) consume<GT, VEC, MAXE>(p, f, raw[k], e0 + k);
+        }
+        for (; e0 < E; ++e0) {                           // fewer than K left
+            Raw<GT, VEC> r;
+            load_raw(r, p.g[e0], i);
+            consume<GT, VEC, MAXE>(p, f, r, e0);
         }
     }
     store_state<VEC>(p.w + first, f.w);

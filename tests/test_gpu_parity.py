@@ -288,6 +288,50 @@ def test_bf16_pull_needs_a_mirror():
     ps.destroy()
 
 
+def test_contiguous_shards_need_no_synchronisation():
+    """The paper shards its parameter server and the shards never talk to each other (Section 2.3).
+    Three servers over contiguous ranges of one vector, fed the same pushes, give bit for bit the
+    state of one server over the whole vector, and their clocks and logs stay in lock-step."""
+    dev = torch.device("cuda", 0)
+    n_el, lam, n = 100003, 6, 2
+    bounds = [0, 33336, 70004, n_el]                       # ragged, differently aligned shard starts
+    kinds, learners = R.simulate_arrivals("lognormal", lam, 60, 14)
+    w0 = G.initial_weights(layouts.flat(n_el), 14).to(dev)
+    whole = P.ParameterServer(n_el, lam, n, 0.02, 0.9, 5e-4, fuse_t=2, device=dev)
+    whole.init_weights(w0)
+    wbuf, vbuf = torch.empty(n_el, device=dev), torch.empty(n_el, device=dev)
+    shards = []
+    for a, b in zip(bounds[:-1], bounds[1:]):
+        sh = P.ParameterServer(b - a, lam, n, 0.02, 0.9, 5e-4, fuse_t=2, device=dev, state=(wbuf[a:b], vbuf[a:b]))
+        sh.init_weights(w0[a:b].contiguous())
+        shards.append((a, b, sh))
+    pulled, counts = {}, {}
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == 0:
+            pulled[l] = whole.pull_weights()
+            assert all(sh.pull_weights() == pulled[l] for _, _, sh in shards)
+            continue
+        c_ = counts.get(l, 0); counts[l] = c_ + 1
+        g = G.gradient(14, l, c_, n_el, 1e-3, device=dev)
+        whole.push_gradient(l, g, pulled[l])
+        for a, b, sh in shards:
+            sh.push_gradient(l, g[a:b], pulled[l])         # slice a of the same gradient goes to shard a
+        if whole.timestamps()[1] - whole.timestamps()[0] >= 2:
+            whole.apply_update()
+            for _, _, sh in shards:
+                sh.apply_update()
+    whole.flush()
+    for _, _, sh in shards:
+        sh.flush()
+    torch.cuda.synchronize()
+    assert torch.equal(whole.w, wbuf) and torch.equal(whole.v, vbuf)
+    for _, _, sh in shards:
+        assert sh.timestamps() == whole.timestamps()
+        assert np.array_equal(sh.update_log(), whole.update_log())
+        sh.destroy()
+    whole.destroy()
+
+
 def test_zero_parameters():
     _simple(0, 4, 2, 12)
 

@@ -197,6 +197,17 @@ int ps_get_update_log(ps_t *ps, int64_t first_update, int64_t count, ps_log_entr
 int ps_peek_state(ps_t *ps, const float **w_dev, const float **v_dev,
                   int64_t *ts_applied, int64_t *ts_logical);
 
+/* Checkpoint of the protocol state (the paper describes none; long trainings need one): timestamp,
+ * current alpha0 and every learner's push count, as PS_STATE_WORDS(lambda) 64-bit words in host memory.
+ * Theta and v are the caller's buffers and are saved by the caller.  Pending gradients are borrowed
+ * device buffers and cannot be saved: both calls return PS_ERR_NOT_READY unless no gradient is waiting
+ * (checkpoint on a group boundary, after ps_flush).  ps_export_state returns the number of words written;
+ * ps_import_state needs a handle created with the same num_params, lambda and n, restarts the log at the
+ * imported timestamp, and leaves theta and v alone. */
+#define PS_STATE_WORDS(lambda) (8 + (lambda))
+int ps_export_state(ps_t *ps, int64_t *out_host, int64_t capacity_words);
+int ps_import_state(ps_t *ps, const int64_t *in_host, int64_t words);
+
 /* With PS_OPT_TIMING = 1: waits for the stream, then returns the summed CUDA-event duration of the
  * update kernels launched since the last call and their number.  Either pointer may be NULL. */
 int ps_kernel_time(ps_t *ps, double *total_ms, int64_t *launches);

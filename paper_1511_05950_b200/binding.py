@@ -42,7 +42,7 @@ EXPORTS = (
     "ps_pull_weights_bf16",
     "ps_set_option", "ps_get_option", "ps_set_alpha0", "ps_pull_weights", "ps_pull_weights_host", "ps_pull_weights_host_async",
     "ps_push_gradient", "ps_push_gradient_host", "ps_apply_update", "ps_flush", "ps_synchronize",
-    "ps_get_update_log", "ps_peek_state", "ps_kernel_time", "ps_last_cuda_error", "ps_status_string",
+    "ps_get_update_log", "ps_peek_state", "ps_export_state", "ps_import_state", "ps_kernel_time", "ps_last_cuda_error", "ps_status_string",
 )
 
 
@@ -81,6 +81,8 @@ def _load() -> C.CDLL:
         "ps_synchronize": [vp],
         "ps_get_update_log": [vp, i64, i64, vp],
         "ps_peek_state": [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), C.POINTER(i64)],
+        "ps_export_state": [vp, vp, i64],
+        "ps_import_state": [vp, vp, i64],
         "ps_kernel_time": [vp, C.POINTER(C.c_double), C.POINTER(i64)],
         "ps_last_cuda_error": [vp],
         "ps_status_string": [i32],
@@ -117,6 +119,8 @@ ps_synchronize = lib.ps_synchronize
 ps_get_update_log = lib.ps_get_update_log
 ps_peek_state = lib.ps_peek_state
 ps_kernel_time = lib.ps_kernel_time
+ps_export_state = lib.ps_export_state
+ps_import_state = lib.ps_import_state
 ps_last_cuda_error = lib.ps_last_cuda_error
 
 
@@ -148,6 +152,7 @@ class ParameterServer:
                  state: Optional[Tuple[torch.Tensor, torch.Tensor]] = None, allocate: bool = True):
         self._h = C.c_void_p()
         self.num_params = int(num_params)
+        self.num_learners = int(num_learners)
         self.c = num_learners // n if n >= 1 else 0
         self.grad_dtype = grad_dtype
         self._held = collections.deque()
@@ -228,26 +233,34 @@ class ParameterServer:
 
     # -- the protocol ----------------------------------------------------------
     def pull_weights(self, out: Optional[torch.Tensor] = None, non_blocking: bool = False) -> int:
-        """Timestamp a gradient computed from now on must carry; fills `out` with the weights if given.
+        """Timestamp a gradient computed from now on must carry; fills `out` with the weights if given
+        (fp32 on the device or the host, or bf16 on the device when a mirror is bound).
         non_blocking (host `out` only): return once the copy is enqueued; call synchronize() before reading."""
         ts = C.c_int64()
-        if out is not None and out.dtype == torch.bfloat16:
-            assert out.is_cuda and out.is_contiguous()
-            _check(ps_pull_weights_bf16(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_bf16")
-            self._held.clear()
+        if out is None:
+            _check(ps_pull_weights(self._h, None, C.byref(ts)), "ps_pull_weights")
             return ts.value
-        if out is not None and not out.is_cuda:
-            assert out.dtype == torch.float32 and out.is_contiguous()
-            if non_blocking:
-                _check(ps_pull_weights_host_async(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host_async")
-            else:
-                _check(ps_pull_weights_host(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host")
-            self._held.clear()
+        assert out.is_contiguous()
+        applied_before = self.timestamps()[0]
+        if out.dtype == torch.bfloat16:
+            assert out.is_cuda
+            _check(ps_pull_weights_bf16(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_bf16")
+        elif out.is_cuda:
+            assert out.dtype == torch.float32
+            _check(ps_pull_weights(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights")
+        elif non_blocking:
+            assert out.dtype == torch.float32
+            _check(ps_pull_weights_host_async(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host_async")
         else:
-            _check(ps_pull_weights(self._h, _ptr(out), C.byref(ts)), "ps_pull_weights")
-            if out is not None:
-                self._held.clear()
+            assert out.dtype == torch.float32
+            _check(ps_pull_weights_host(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host")
+        self._release(self.timestamps()[0] - applied_before)     # the pull applied every complete group first
         return ts.value
+
+    def _release(self, groups: int) -> None:
+        """Drop the references to the gradients of `groups` applied groups (oldest first)."""
+        for _ in range(groups * self.c):
+            self._held.popleft()
 
     def push_gradient(self, learner: int, grad: torch.Tensor, ts: int) -> bool:
         """True if this push completed a group of c (an update can be applied)."""
@@ -264,14 +277,12 @@ class ParameterServer:
 
     def apply_update(self) -> int:
         done = _check(ps_apply_update(self._h), "ps_apply_update")
-        for _ in range(done * self.c):
-            self._held.popleft()
+        self._release(done)
         return done
 
     def flush(self) -> int:
         done = _check(ps_flush(self._h), "ps_flush")
-        for _ in range(done * self.c):
-            self._held.popleft()
+        self._release(done)
         return done
 
     def synchronize(self) -> None:
@@ -292,6 +303,19 @@ class ParameterServer:
         _check(ps_get_update_log(self._h, first_update, count, out.ctypes.data if out.size else None),
                "ps_get_update_log")
         return out
+
+    def export_state(self) -> np.ndarray:
+        """Protocol state (timestamp, rate, push counts) as int64 words; weights and momentum are self.w, self.v."""
+        out = np.empty(8 + len(self._learners()), dtype=np.int64)
+        n = _check(ps_export_state(self._h, out.ctypes.data, out.size), "ps_export_state")
+        return out[:n].copy()
+
+    def import_state(self, words: np.ndarray) -> None:
+        words = np.ascontiguousarray(words, dtype=np.int64)
+        _check(ps_import_state(self._h, words.ctypes.data, words.size), "ps_import_state")
+
+    def _learners(self):
+        return range(self.num_learners)
 
     def kernel_time(self) -> Tuple[float, int]:
         ms, n = C.c_double(), C.c_int64()

@@ -7,6 +7,7 @@
 #include "update_kernels.cuh"
 
 #include <algorithm>
+#include <cstring>
 #include <deque>
 #include <mutex>
 #include <new>
@@ -627,6 +628,49 @@ int ps_peek_state(ps_t *ps, const float **w_dev, const float **v_dev, int64_t *t
     if (v_dev) *v_dev = ps->v;
     if (ts_applied) *ts_applied = ps->ts_applied;
     if (ts_log) *ts_log = ts_logical(ps);
+    return PS_OK;
+}
+
+namespace {
+constexpr int64_t kStateMagic = 0x5053534F46545359LL;   // "PSSOFTSY"
+constexpr int64_t kStateVersion = 1;
+constexpr int64_t kStateHeader = 8;
+}  // namespace
+
+int ps_export_state(ps_t *ps, int64_t *out_host, int64_t capacity_words)
+{
+    if (!is_live(ps) || !out_host) return PS_ERR_INVALID_ARG;
+    const int64_t words = kStateHeader + ps->lambda;
+    if (capacity_words < words) return PS_ERR_INVALID_ARG;
+    if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_NOT_READY;   // borrowed gradients cannot be saved
+    uint32_t alpha_bits;
+    static_assert(sizeof alpha_bits == sizeof ps->alpha0, "fp32 rate");
+    std::memcpy(&alpha_bits, &ps->alpha0, sizeof alpha_bits);
+    out_host[0] = kStateMagic; out_host[1] = kStateVersion;
+    out_host[2] = ps->n; out_host[3] = ps->lambda; out_host[4] = ps->split;
+    out_host[5] = ps->ts_applied; out_host[6] = static_cast<int64_t>(alpha_bits); out_host[7] = ps->launches;
+    for (int l = 0; l < ps->lambda; ++l) out_host[kStateHeader + l] = ps->push_count[l];
+    return static_cast<int>(words);
+}
+
+int ps_import_state(ps_t *ps, const int64_t *in_host, int64_t words)
+{
+    if (!is_live(ps) || !in_host || words < kStateHeader) return PS_ERR_INVALID_ARG;
+    if (in_host[0] != kStateMagic || in_host[1] != kStateVersion) return PS_ERR_INVALID_ARG;
+    if (in_host[2] != ps->n || in_host[3] != ps->lambda || in_host[4] != ps->split) return PS_ERR_INVALID_ARG;
+    if (words != kStateHeader + ps->lambda || in_host[5] < 0 || in_host[7] < 0) return PS_ERR_INVALID_ARG;
+    for (int l = 0; l < ps->lambda; ++l) if (in_host[kStateHeader + l] < 0) return PS_ERR_INVALID_ARG;
+    if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_NOT_READY;
+    const uint32_t alpha_bits = static_cast<uint32_t>(in_host[6]);
+    float alpha0;
+    std::memcpy(&alpha0, &alpha_bits, sizeof alpha0);
+    if (!(alpha0 == alpha0)) return PS_ERR_INVALID_ARG;
+    ps->alpha0 = alpha0;
+    ps->ts_applied = in_host[5];
+    ps->launches = in_host[7];
+    for (int l = 0; l < ps->lambda; ++l) ps->push_count[l] = in_host[kStateHeader + l];
+    ps->log.clear();
+    ps->log_first_update = ps->ts_applied;
     return PS_OK;
 }
 

@@ -214,6 +214,53 @@ def test_weight_mirror_argument_checks():
     P.ps_destroy(h)
 
 
+def test_checkpoint_on_a_group_boundary_resumes_the_same_schedule():
+    lam, n, pushes = 6, 2, 120
+    c = lam // n
+    kinds, learners = R.simulate_arrivals("lognormal", lam, pushes, 77)
+    ref = R.ReferencePS(0, lam, n, 0.01, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(np.zeros(0, np.float32))
+    nothing = np.zeros(0, np.float32)
+    rc, h = make(lam, n)
+    pulled, ts, done, cut = {}, C.c_int64(), 0, None
+    words = np.empty(8 + lam, dtype=np.int64)
+    for i, (k, l) in enumerate(zip(kinds.tolist(), learners.tolist())):
+        if k == PULL:
+            ref.pull(l)
+            assert P.ps_pull_weights(h, None, C.byref(ts)) == 0
+            pulled[l] = ts.value
+            continue
+        ref.push(l, nothing)
+        if cut is None and done == 58 and done % c != 0:
+            assert P.ps_export_state(h, words.ctypes.data, words.size) == P.PS_ERR_NOT_READY    # mid-group
+        r = P.ps_push_gradient(h, l, FAKE_GRAD, pulled[l])
+        done += 1
+        if r == P.PS_READY:
+            assert P.ps_apply_update(h) == 1
+            if cut is None and done >= 60:
+                if done == 60:
+                    P.ps_set_alpha0(h, 0.005); ref.set_alpha0(0.005)
+                assert P.ps_export_state(h, words.ctypes.data, 3) == P.PS_ERR_INVALID_ARG      # too small
+                assert P.ps_export_state(h, words.ctypes.data, words.size) == 8 + lam
+                cut = done // c
+                assert P.ps_destroy(h) == 0
+                rc, h = make(lam, n)                                    # a new server takes over
+                bad = words.copy(); bad[3] = lam + 1
+                assert P.ps_import_state(h, bad.ctypes.data, bad.size) == P.PS_ERR_INVALID_ARG
+                assert P.ps_import_state(h, words.ctypes.data, words.size - 1) == P.PS_ERR_INVALID_ARG
+                assert P.ps_import_state(h, words.ctypes.data, words.size) == 0
+                assert P.ps_peek_state(h, None, None, C.byref(ts), None) == 0 and ts.value == cut
+    n_upd = pushes // c
+    out = np.empty((n_upd - cut) * c, dtype=P.binding.LOG_DTYPE)
+    assert P.ps_get_update_log(h, cut, n_upd - cut, out.ctypes.data) == 0
+    assert P.ps_get_update_log(h, cut - 1, 1, out.ctypes.data) == P.PS_ERR_LOG_EVICTED          # log restarts at the cut
+    rlog = ref.log()[cut * c:]
+    for f in ("update", "push_index", "ts_grad", "tau", "sigma", "learner", "position"):
+        assert np.array_equal(out[f], rlog[f]), f
+    assert np.array_equal(out["scale"], rlog["scale"].astype(np.float32))
+    P.ps_destroy(h)
+
+
 def test_status_strings():
     assert P.status_string(P.PS_ERR_BAD_TIMESTAMP).startswith("gradient timestamp")
     assert P.status_string(0) == "ok"

@@ -332,6 +332,46 @@ def test_contiguous_shards_need_no_synchronisation():
     whole.destroy()
 
 
+def test_checkpoint_and_resume_reproduce_the_uninterrupted_run():
+    """Save theta, v and the exported protocol state on a group boundary, restore them into a fresh server,
+    carry on: the final state equals the reference's uninterrupted run bit for bit."""
+    from tests.gpu_harness import as_reference_grad
+    dev = torch.device("cuda", 0)
+    n_el, lam, n = 40009, 4, 2
+    kinds, learners = R.simulate_arrivals("exp", lam, 64, 21)
+    w0 = G.initial_weights(layouts.flat(n_el), 21)
+    ref = R.ReferencePS(n_el, lam, n, 0.03, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    ps = P.ParameterServer(n_el, lam, n, 0.03, 0.9, 5e-4, device=dev)
+    ps.init_weights(w0.to(dev))
+    pulled, counts, pushes, resumed = {}, {}, 0, False
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == 0:
+            pulled[l] = ps.pull_weights()
+            assert ref.pull(l) == pulled[l]
+            continue
+        b = counts.get(l, 0); counts[l] = b + 1
+        g = G.gradient(21, l, b, n_el, 1e-3, device=dev)
+        ref.push(l, as_reference_grad(g))
+        if ps.push_gradient(l, g, pulled[l]):
+            ps.apply_update()
+        pushes += 1
+        if pushes == 30 and not resumed:
+            ps.synchronize()
+            saved = (ps.w.clone(), ps.v.clone(), ps.export_state())
+            ps.destroy()
+            ps = P.ParameterServer(n_el, lam, n, 0.03, 0.9, 5e-4, device=dev)
+            ps.w.copy_(saved[0]); ps.v.copy_(saved[1])
+            ps.import_state(saved[2])
+            assert ps.timestamps() == (15, 15)
+            resumed = True
+    ps.flush(); ps.synchronize()
+    w, v = ref.state()
+    assert np.array_equal(ps.w.cpu().numpy(), w.astype(np.float32)) and np.array_equal(ps.v.cpu().numpy(), v.astype(np.float32))
+    assert np.array_equal(ps.update_log(15)["tau"], ref.log()["tau"][30:])
+    ps.destroy()
+
+
 def test_zero_parameters():
     _simple(0, 4, 2, 12)
 

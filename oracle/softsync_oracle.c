@@ -15,7 +15,7 @@
  *   - each gradient is scaled by alpha0 / tau when tau > 0 (Eq. 3) or by the
  *     constant alpha0 (the control experiment of Section 4.3).
  *
- * Readings where the paper is silent (all listed in the design notes):
+ * Readings where the paper is silent:
  *   - tau = 0 is given the full alpha0: sigma = max(tau, 1).  Eq. 1 (hardsync,
  *     tau = 0) uses the full learning rate.
  *   - an update takes exactly c gradients, first come first grouped.

@@ -110,3 +110,49 @@ def test_large_stale_bf16_full_size():
     """Config 4: same vector, lambda=54, n=54 (c=1), bf16 gradients, 2,000 pushes applied 8 per pass."""
     log = run_full(configs.LARGE_STALE_BF16, lazy=True)
     assert len(log) == 2000 and log["tau"].max() > 100
+
+
+@pytest.mark.parametrize("grad_dtype", ["fp32", "bf16"])
+def test_more_than_two_to_the_thirty_elements(grad_dtype):
+    """A ragged vector of 2^30 + 3 elements (the sweep's largest size): byte offsets beyond 2^32, the
+    scalar tail after the last full fragment, both traversal directions.  Sampled parity over 3 updates."""
+    from workloads import layouts
+    dev = torch.device("cuda", 0)
+    n = (1 << 30) + 3
+    need = n * (8 + 2 * 4) + (6 << 30)
+    free, _ = torch.cuda.mem_get_info(dev)
+    if free < need:
+        pytest.skip("not enough free device memory for the 2^30-element case")
+    tdt = TORCH_DTYPE[grad_dtype]
+    layout = layouts.flat(n)
+    rng = np.random.default_rng(5)
+    picks = set(rng.integers(0, n, size=3000).tolist())
+    for centre in (0, 1 << 29, (1 << 30) - 64, 1 << 30, n - 1):
+        picks.update(k for k in range(centre - 40, centre + 40) if 0 <= k < n)
+    idx = torch.tensor(sorted(picks), dtype=torch.int64)
+    idx_dev = idx.to(dev)
+    lam, c = 2, 2
+    ref = R.ReferencePS(idx.numel(), lam, 1, 0.01, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(G.initial_weights_at(layout, 3, idx).numpy())
+    ps = P.ParameterServer(n, lam, 1, 0.01, 0.9, 5e-4, grad_dtype=grad_dtype, device=dev)
+    G.normal_like(G.stream_key(3, G.STREAM_WEIGHTS), 0, n, 0.01, out=ps.w)
+    ps.v.zero_()
+    for u in range(3):
+        grads = []
+        for l in range(lam):
+            ts = ps.pull_weights()
+            assert ref.pull(l) == ts
+        for l in range(lam):
+            g = torch.empty(n, dtype=tdt, device=dev)
+            G.gradient(3, l, u, n, 1e-3, dtype=tdt, device=dev, out=g)
+            grads.append(g)
+            ref.push(l, as_reference_grad(G.gradient_at(3, l, u, idx, 1e-3, dtype=tdt)))
+            ps.push_gradient(l, g, u)
+        assert ps.apply_update() == 1
+        ps.synchronize()
+        del grads
+    w32, v32 = ref.state()
+    assert np.array_equal(ps.w[idx_dev].cpu().numpy(), w32.astype(np.float32))
+    assert np.array_equal(ps.v[idx_dev].cpu().numpy(), v32.astype(np.float32))
+    assert ps.timestamps() == (3, 3)
+    ps.destroy()

@@ -158,6 +158,12 @@ def step_events(cfg, num_steps: int):
 
 # ----------------------------------------------------------------------------- our arm
 def run_ours(args, cfg, rank, world, local_rank):
+    from paper_1511_05950_b200 import build as lib_build
+    if local_rank == 0:
+        lib_build.ensure_built()                   # no-op when the in-tree library is current
+    if world > 1:
+        import torch.distributed as dist_
+        dist_.barrier()
     import paper_1511_05950_b200 as P
     import torch.distributed as dist
 
@@ -300,46 +306,73 @@ TRAFFIC = {"large_softsync": 1.913e9, "large_stale_bf16": 1.913e9}
 
 
 # ----------------------------------------------------------------------------- oracle arms
-def oracle_sample(cfg, sample_params: int, updates: int, rotate: int = 8):
+def oracle_sample(cfg, sample_params: int, updates: int, rotate: int = 8, threads: int = 1):
     """Time the CPU reference, as it stands, on `updates` updates over the first `sample_params`
-    elements of the workload.  Returns (grad elements per second, seconds)."""
+    elements of the workload.  threads > 1: that many unmodified reference servers, each on its own
+    contiguous range of the vector (the update is element-wise, so the result is the same).
+    Returns (grad elements per second, seconds)."""
+    from concurrent.futures import ThreadPoolExecutor
+
     from oracle import reference as R
 
     layout = cfg.layout()
     idx_n = min(sample_params, layout.num_params)
     gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
     tdt = torch.bfloat16 if cfg.grad_dtype == "bf16" else torch.float32
-    w0 = G.initial_weights(layout, cfg.seed, cfg.weight_std, device=gen_dev)[:idx_n].cpu()
+    w0 = G.initial_weights(layout, cfg.seed, cfg.weight_std, device=gen_dev)[:idx_n].cpu().numpy()
     grads = []
     for i in range(rotate):
         g = G.gradient(cfg.seed, i, 0, idx_n, cfg.grad_std, dtype=tdt, device=gen_dev).cpu()
         grads.append(g.view(torch.int16).numpy().view(np.uint16) if tdt == torch.bfloat16 else g.numpy())
-    ref = R.ReferencePS(idx_n, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
-                        R.MOD_INV_STALENESS if cfg.modulation == "inv_staleness" else R.MOD_CONSTANT, 32)
-    ref.set_weights(w0.numpy())
+    threads = max(1, min(threads, idx_n))
+    bounds = [idx_n * t // threads for t in range(threads + 1)]
+    mod = R.MOD_INV_STALENESS if cfg.modulation == "inv_staleness" else R.MOD_CONSTANT
+    servers = []
+    for a, b in zip(bounds[:-1], bounds[1:]):
+        ref = R.ReferencePS(b - a, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay, mod, 32)
+        ref.set_weights(w0[a:b])
+        servers.append((a, b, ref))
     steps = step_events(cfg, updates)
-    i = 0
+
+    def replay(part):
+        a, b, ref = part
+        i = 0
+        for evs in steps:
+            for k, l in evs:
+                if k == arrivals.PULL:
+                    ref.pull(l)
+                else:
+                    ref.push(l, grads[i % rotate][a:b])          # ctypes calls release the GIL
+                    i += 1
+        return ref.timestamp
+
     t0 = time.perf_counter()
-    for evs in steps:
-        for k, l in evs:
-            if k == arrivals.PULL:
-                ref.pull(l)
-            else:
-                ref.push(l, grads[i % rotate])
-                i += 1
+    if threads == 1:
+        done = [replay(servers[0])]
+    else:
+        with ThreadPoolExecutor(threads) as pool:
+            done = list(pool.map(replay, servers))
     dt = time.perf_counter() - t0
-    assert ref.timestamp == updates
+    assert all(d == updates for d in done)
     return cfg.c * idx_n * updates / dt, dt
 
 
 def cpu_baseline(cfg):
     # about 10 s of single-thread work at the reference's ~6e8 gradient elements/s, at most the whole workload
-    per_update_s = cfg.c * cfg.layout().num_params / 6e8
+    n = cfg.layout().num_params
+    per_update_s = cfg.c * n / 6e8
     updates = int(max(24, min(cfg.num_updates, 10.0 / per_update_s)))
-    v, dt = oracle_sample(cfg, cfg.layout().num_params, updates)
-    return {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": "first %d updates of the workload at full size (%d parameters), fp32 reference, "
-                      "single thread, %.1f s; host has %d cores" % (updates, cfg.layout().num_params, dt, os.cpu_count())}
+    v, dt = oracle_sample(cfg, n, updates)
+    cores = os.cpu_count() or 1
+    out = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": "first %d updates of the workload at full size (%d parameters), fp32 reference, "
+                     "single thread, %.1f s; host has %d cores" % (updates, n, dt, cores)}
+    if cores > 1 and n >= (1 << 20):
+        va, dta = oracle_sample(cfg, n, updates, threads=cores)
+        out["all_cores"] = {"value": va, "unit": UNIT, "cores": cores,
+                            "sample": "same updates, %d unmodified reference servers on contiguous ranges of the "
+                                      "vector, one thread each, %.1f s" % (cores, dta)}
+    return out
 
 
 def run_reference(args, cfg):
@@ -362,6 +395,12 @@ def run_reference(args, cfg):
 
 
 def run_sweep(args):
+    from paper_1511_05950_b200 import build as lib_build
+    lib_build.ensure_built()
+    return _run_sweep(args)
+
+
+def _run_sweep(args):
     """Bandwidth sweep: flat fp32 vectors of 1M .. 1B parameters, c in {1,4,16,64}, fp32 and bf16
     gradients, staleness uniform in [1, 2c], 50 updates per point after 5 warm-up updates."""
     import paper_1511_05950_b200 as P

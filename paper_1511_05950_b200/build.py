@@ -39,6 +39,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def ensure_built() -> str:
+    """Build the library if it is missing or older than its sources.  A stale library is kept when the
+    rebuild fails (no compiler on this machine); a missing one is an error."""
+    if not os.path.exists(LIB):
+        return build(force=True)
+    if is_stale():
+        try:
+            return build(force=True)
+        except Exception:
+            return LIB
+    return LIB
+
+
 if __name__ == "__main__":
     import sys
     print(build(force=True, verbose="-v" in sys.argv))

@@ -10,6 +10,11 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200)")
+    # the C-ABI library and the C reference are built in-tree; (re)build them when missing or out of date
+    from paper_1511_05950_b200 import build as lib_build
+    lib_build.ensure_built()
+    from oracle import build as oracle_build
+    oracle_build.build()
 
 
 def pytest_collection_modifyitems(config, items):

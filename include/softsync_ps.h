@@ -46,7 +46,8 @@ enum ps_status {
     PS_ERR_CUDA = -6,                     /* a CUDA call failed; see ps_last_cuda_error */
     PS_ERR_NOMEM = -7,                    /* host allocation failed */
     PS_ERR_NO_STATE = -8,                 /* weights/momentum (or staging slots) not bound yet */
-    PS_ERR_LOG_EVICTED = -9               /* requested log range is no longer (or not yet) held */
+    PS_ERR_LOG_EVICTED = -9,              /* requested log range is no longer (or not yet) held */
+    PS_ERR_BARRIER = -10                  /* hardsync: this learner has already contributed to the current round */
 };
 
 enum ps_grad_dtype { PS_GRAD_FP32 = 0, PS_GRAD_BF16 = 1 };
@@ -59,6 +60,7 @@ enum ps_option {
     PS_OPT_LOG_UPDATES = 5,               /* how many most recent updates the log keeps (default 65536) */
     PS_OPT_TIMING = 6,                    /* 1: bracket every update kernel with CUDA events (ps_kernel_time) */
     PS_OPT_KERNEL = 7,                    /* ps_kernel_choice (default PS_KERNEL_AUTO) */
+    PS_OPT_PROTOCOL = 10,                 /* ps_protocol (default PS_PROTOCOL_SOFTSYNC); only while nothing is pending */
     PS_OPT_OVERLAP_LAUNCH = 9,            /* 1: update kernels are launched as programmatic dependents (see below); default 0 */
     PS_OPT_BLOCK_THREADS = 8              /* threads per block: 128, 256 or 512; 0 = default (128) */
 };
@@ -69,6 +71,15 @@ enum ps_option {
  * directly precedes a ps_apply_update on the server's stream and may still be running (gradients written
  * by earlier kernels, by kernels the host has already synchronised with, by copies, or on other streams
  * with proper ordering are fine).  Results are bit-identical either way. */
+
+/* Section 2.2 describes two protocols.  n-softsync (the default): an update after c = floor(lambda/n)
+ * gradients from any learners, stale gradients welcome.  Hardsync (Eq. 1, synchronous SGD): one update per
+ * round from exactly one gradient of every learner, all computed on the current weights.  In hardsync mode
+ * (needs n = 1, so c = lambda) ps_push_gradient enforces the barrier: a gradient whose timestamp is not the
+ * server's current one is refused with PS_ERR_BAD_TIMESTAMP (staleness must be 0), a second gradient from a
+ * learner within one round with PS_ERR_BARRIER.  The update itself is the same kernel: Eq. 2 with all
+ * staleness 0 is Eq. 1. */
+enum ps_protocol { PS_PROTOCOL_SOFTSYNC = 0, PS_PROTOCOL_HARDSYNC = 1 };
 
 enum ps_kernel_choice {
     PS_KERNEL_AUTO = 0,                   /* vector kernel when every pointer is 16-byte aligned, else scalar */

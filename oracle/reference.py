@@ -39,6 +39,7 @@ def load(path: str) -> C.CDLL:
         L.oracle_ps_destroy.argtypes = [C.c_void_p]
         L.oracle_ps_set_weights.argtypes = [C.c_void_p, C.c_void_p]
         L.oracle_ps_set_alpha0.argtypes = [C.c_void_p, C.c_float]
+        L.oracle_ps_set_hardsync.argtypes = [C.c_void_p, C.c_int]
         L.oracle_ps_timestamp.restype = C.c_int64
         L.oracle_ps_timestamp.argtypes = [C.c_void_p]
         L.oracle_ps_group_size.argtypes = [C.c_void_p]
@@ -121,6 +122,11 @@ class ReferencePS:
         w0 = np.ascontiguousarray(w0, dtype=np.float32)
         assert w0.size == self.num_params
         lib().oracle_ps_set_weights(self._h, w0.ctypes.data)
+
+    def set_hardsync(self, on: bool = True) -> None:
+        """Switch to the hardsync protocol (needs n = 1, nothing pending)."""
+        if lib().oracle_ps_set_hardsync(self._h, int(on)) != 0:
+            raise ValueError("hardsync needs n = 1 and no pending gradient")
 
     def set_alpha0(self, alpha0: float) -> None:
         """Base learning rate for gradients pushed from now on."""

@@ -87,6 +87,7 @@ typedef struct {
 typedef struct oracle_ps {
     int64_t N;
     int lambda, n, c, modulation, precision;
+    int hardsync;                    /* 1: the hardsync protocol of Section 2.2 (barrier, staleness 0) */
     double alpha0, momentum, wd;     /* exact widenings of the fp32 parameters */
     void *w, *v;
     int64_t ts;
@@ -137,6 +138,17 @@ void oracle_ps_set_weights(oracle_ps *ps, const float *w0)
         else { ((double *)ps->w)[k] = (double)w0[k]; ((double *)ps->v)[k] = 0.0; }
     }
     ps->ts = 0;
+}
+
+/* Hardsync protocol (Section 2.2, Eq. 1): the server waits for one gradient from every learner, all
+ * computed on the current weights, averages them and updates; needs n = 1 so that c = lambda.
+ * Returns 0, or -1 if n != 1 or gradients are pending. */
+int oracle_ps_set_hardsync(oracle_ps *ps, int on)
+{
+    if (on && ps->n != 1) return -1;
+    if (ps->npending) return -1;
+    ps->hardsync = on ? 1 : 0;
+    return 0;
 }
 
 /* Learning-rate schedule: the base rate for gradients that arrive from now on (Section 4.3). */
@@ -221,6 +233,11 @@ int oracle_ps_push_with_timestamp(oracle_ps *ps, int learner, const void *grad, 
     if (j < 0) return -2;
     const int64_t tau = ps->ts - j;                      /* staleness, Section 2.1 */
     if (tau < 0) return -3;
+    if (ps->hardsync) {
+        if (tau != 0) return -3;                         /* "ensures that the gradient staleness is 0" */
+        for (int q = 0; q < ps->npending; ++q)           /* one contribution per learner and round */
+            if (ps->pending[q].learner == learner) return -4;
+    }
     int64_t sigma = 1;
     if (ps->modulation == ORACLE_MOD_INV_STALENESS)
         sigma = tau > 0 ? tau : 1;                       /* Eq. 3, and alpha0 itself at tau = 0 */

@@ -22,10 +22,11 @@ from . import build as _build
 PS_MOD_CONSTANT, PS_MOD_INV_STALENESS = 0, 1
 PS_OK, PS_READY = 0, 1
 PS_ERR_INVALID_ARG, PS_ERR_BAD_LEARNER, PS_ERR_BAD_TIMESTAMP, PS_ERR_NOT_READY = -1, -2, -3, -4
-PS_ERR_QUEUE_FULL, PS_ERR_CUDA, PS_ERR_NOMEM, PS_ERR_NO_STATE, PS_ERR_LOG_EVICTED = -5, -6, -7, -8, -9
+PS_ERR_QUEUE_FULL, PS_ERR_CUDA, PS_ERR_NOMEM, PS_ERR_NO_STATE, PS_ERR_LOG_EVICTED, PS_ERR_BARRIER = -5, -6, -7, -8, -9, -10
 PS_GRAD_FP32, PS_GRAD_BF16 = 0, 1
 (PS_OPT_GRAD_DTYPE, PS_OPT_FUSE_T, PS_OPT_STREAM, PS_OPT_QUEUE_GROUPS, PS_OPT_LOG_UPDATES,
- PS_OPT_TIMING, PS_OPT_KERNEL, PS_OPT_BLOCK_THREADS, PS_OPT_OVERLAP_LAUNCH) = range(1, 10)
+ PS_OPT_TIMING, PS_OPT_KERNEL, PS_OPT_BLOCK_THREADS, PS_OPT_OVERLAP_LAUNCH, PS_OPT_PROTOCOL) = range(1, 11)
+PS_PROTOCOL_SOFTSYNC, PS_PROTOCOL_HARDSYNC = 0, 1
 PS_KERNEL_AUTO, PS_KERNEL_SCALAR, PS_KERNEL_VECTOR = 0, 1, 2
 PS_MAX_GROUP, PS_MAX_FUSE_T, PS_MAX_ENTRIES = 256, 16, 512
 

@@ -52,6 +52,7 @@ struct ps_ctx {
     int64_t queue_groups = 64;
     int64_t log_updates = 65536;
     int timing = 0, kernel_choice = PS_KERNEL_AUTO, block_threads = 0, overlap_launch = 0;
+    int protocol = PS_PROTOCOL_SOFTSYNC;
     int sm_count = 0;
 
     int64_t ts_applied = 0;                // updates whose kernel has been enqueued
@@ -314,6 +315,11 @@ int check_push(ps_ctx *ps, int learner, const void *grad, int64_t ts)
     if (!grad && ps->n > 0) return PS_ERR_INVALID_ARG;    // a zero-length gradient has no address
     if (learner < 0 || learner >= ps->lambda) return PS_ERR_BAD_LEARNER;
     if (ts < 0 || ts > ts_logical(ps)) return PS_ERR_BAD_TIMESTAMP;
+    if (ps->protocol == PS_PROTOCOL_HARDSYNC) {           // Section 2.2: everybody works on the current weights
+        if (ts != ts_logical(ps)) return PS_ERR_BAD_TIMESTAMP;
+        for (const Entry &en : ps->filling)
+            if (en.learner == learner) return PS_ERR_BARRIER;
+    }
     if (static_cast<int64_t>(ps->ready.size()) >= ps->queue_groups) return PS_ERR_QUEUE_FULL;
     return PS_OK;
 }
@@ -463,6 +469,11 @@ int ps_set_option(ps_t *ps, int key, int64_t value)
     case PS_OPT_KERNEL:
         if (value < PS_KERNEL_AUTO || value > PS_KERNEL_VECTOR) return PS_ERR_INVALID_ARG;
         ps->kernel_choice = static_cast<int>(value); return PS_OK;
+    case PS_OPT_PROTOCOL:
+        if (value != PS_PROTOCOL_SOFTSYNC && value != PS_PROTOCOL_HARDSYNC) return PS_ERR_INVALID_ARG;
+        if (value == PS_PROTOCOL_HARDSYNC && ps->split != 1) return PS_ERR_INVALID_ARG;
+        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+        ps->protocol = static_cast<int>(value); return PS_OK;
     case PS_OPT_OVERLAP_LAUNCH:
         if (value != 0 && value != 1) return PS_ERR_INVALID_ARG;
         ps->overlap_launch = static_cast<int>(value); return PS_OK;
@@ -487,6 +498,7 @@ int ps_get_option(ps_t *ps, int key, int64_t *value)
     case PS_OPT_KERNEL: *value = ps->kernel_choice; return PS_OK;
     case PS_OPT_BLOCK_THREADS: *value = ps->block_threads; return PS_OK;
     case PS_OPT_OVERLAP_LAUNCH: *value = ps->overlap_launch; return PS_OK;
+    case PS_OPT_PROTOCOL: *value = ps->protocol; return PS_OK;
     default: return PS_ERR_INVALID_ARG;
     }
 }
@@ -709,6 +721,7 @@ const char *ps_status_string(int status)
     case PS_ERR_NOMEM: return "host allocation failed";
     case PS_ERR_NO_STATE: return "weights, momentum or staging slots not bound";
     case PS_ERR_LOG_EVICTED: return "log range not held";
+    case PS_ERR_BARRIER: return "hardsync: learner already contributed to this round";
     default: return status > 1 ? "updates applied" : "unknown status";
     }
 }

@@ -261,6 +261,30 @@ def test_checkpoint_on_a_group_boundary_resumes_the_same_schedule():
     P.ps_destroy(h)
 
 
+def test_hardsync_mode_enforces_the_barrier():
+    rc, h = make(3, 3)
+    assert P.ps_set_option(h, P.PS_OPT_PROTOCOL, P.PS_PROTOCOL_HARDSYNC) == P.PS_ERR_INVALID_ARG   # needs n = 1
+    P.ps_destroy(h)
+    rc, h = make(3, 1)
+    assert P.ps_set_option(h, P.PS_OPT_PROTOCOL, 2) == P.PS_ERR_INVALID_ARG
+    assert P.ps_set_option(h, P.PS_OPT_PROTOCOL, P.PS_PROTOCOL_HARDSYNC) == 0
+    out = C.c_int64()
+    assert P.ps_get_option(h, P.PS_OPT_PROTOCOL, C.byref(out)) == 0 and out.value == 1
+    for rnd in range(4):
+        assert P.ps_push_gradient(h, 1, FAKE_GRAD, rnd) == P.PS_OK
+        assert P.ps_push_gradient(h, 1, FAKE_GRAD, rnd) == P.PS_ERR_BARRIER        # twice in one round
+        if rnd:
+            assert P.ps_push_gradient(h, 0, FAKE_GRAD, rnd - 1) == P.PS_ERR_BAD_TIMESTAMP   # old weights
+        assert P.ps_push_gradient(h, 0, FAKE_GRAD, rnd) == P.PS_OK
+        assert P.ps_set_option(h, P.PS_OPT_PROTOCOL, 0) == P.PS_ERR_INVALID_ARG   # not in mid-round
+        assert P.ps_push_gradient(h, 2, FAKE_GRAD, rnd) == P.PS_READY
+        assert P.ps_apply_update(h) == 1
+    ts, log = fetch_log(h, 3)
+    assert ts == 4 and (log["tau"] == 0).all() and log["learner"].tolist() == [0, 1, 2] * 4
+    assert P.status_string(P.PS_ERR_BARRIER).startswith("hardsync")
+    P.ps_destroy(h)
+
+
 def test_status_strings():
     assert P.status_string(P.PS_ERR_BAD_TIMESTAMP).startswith("gradient timestamp")
     assert P.status_string(0) == "ok"

@@ -372,6 +372,42 @@ def test_checkpoint_and_resume_reproduce_the_uninterrupted_run():
     ps.destroy()
 
 
+def test_hardsync_protocol_matches_reference():
+    """Eq. 1 through the C ABI: rounds of one gradient per learner on the current weights."""
+    from tests.gpu_harness import as_reference_grad
+    dev = torch.device("cuda", 0)
+    n_el, lam = 33333, 6
+    w0 = G.initial_weights(layouts.flat(n_el), 16)
+    ps = P.ParameterServer(n_el, lam, 1, 0.02, 0.9, 5e-4, device=dev)
+    ps.set_option(P.PS_OPT_PROTOCOL, P.PS_PROTOCOL_HARDSYNC)
+    ps.init_weights(w0.to(dev))
+    refs = {prec: R.ReferencePS(n_el, lam, 1, 0.02, 0.9, 5e-4, R.MOD_INV_STALENESS, prec) for prec in (32, 64)}
+    for r in refs.values():
+        r.set_weights(w0.numpy())
+        r.set_hardsync()
+    for rnd in range(8):
+        ts = ps.pull_weights()
+        assert ts == rnd
+        for r in refs.values():
+            for l in range(lam):
+                r.pull(l)
+        for l in np.random.default_rng(rnd).permutation(lam):
+            g = G.gradient(16, int(l), rnd, n_el, 1e-3, device=dev)
+            for r in refs.values():
+                r.push(int(l), as_reference_grad(g))
+            if ps.push_gradient(int(l), g, ts):
+                ps.apply_update()
+            elif l % 2 == 0:
+                with pytest.raises(P.SoftsyncError) as e:
+                    ps.push_gradient(int(l), g, ts)
+                assert e.value.status == P.PS_ERR_BARRIER
+    ps.synchronize()
+    w, v, log = ps.w.cpu().numpy(), ps.v.cpu().numpy(), ps.update_log()
+    ps.destroy()
+    assert_parity(w, v, log, {prec: (*r.state(), r.log()) for prec, r in refs.items()}, TOL_FP32)
+    assert (log["tau"] == 0).all()
+
+
 def test_zero_parameters():
     _simple(0, 4, 2, 12)
 

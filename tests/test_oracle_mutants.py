@@ -27,6 +27,7 @@ MUTANTS = {
     "wrong_scale_index": ("update_rule.inc", "acc = acc + s[l] * grads[l][k];", "acc = acc + s[0] * grads[l][k];"),
     "decay_unmodulated": ("update_rule.inc", "const REAL d = ROUND_SCALE(wd * S);", "const REAL d = ROUND_SCALE(wd * alpha0[0]);"),
     "rate_at_apply_time": ("softsync_oracle.c", "alpha0[l] = ps->pending[order[l]].alpha0;", "alpha0[l] = ps->alpha0;"),
+    "barrier_lets_stale_in": ("softsync_oracle.c", "if (tau != 0) return -3;", "if (tau > 1) return -3;"),
     "staleness_plus_one": ("softsync_oracle.c", "sigma = tau > 0 ? tau : 1;", "sigma = tau + 1;"),
     "staleness_ignored": ("softsync_oracle.c", "sigma = tau > 0 ? tau : 1;", "sigma = 1;"),
     "clock_jumps": ("softsync_oracle.c", "ps->ts += 1;", "ps->ts += ps->c;"),
@@ -45,6 +46,7 @@ def _pins():
         TU.test_single_learner_matches_library_sgd_optimizer,
         lambda: TU.test_one_softsync_with_barrier_is_synchronous_averaged_sgd(4),
         TU.test_downpour_case_is_per_push_sgd,
+        TU.test_hardsync_protocol_is_eq_1_and_enforces_the_barrier,
         TU.test_step_schedule_without_momentum_is_library_sgd_with_a_changing_rate,
         TU.test_rate_in_force_at_arrival_enters_the_geometric_sum,
         lambda: TU.test_plain_rule_is_a_weighted_sum_of_gradients("exp", 12, 3),
@@ -73,7 +75,7 @@ def test_planted_mistake_is_caught(name, tmp_path):
         for pin in _pins():
             try:
                 pin()
-            except (AssertionError, ValueError):
+            except (AssertionError, ValueError, pytest.fail.Exception):
                 caught += 1
     assert caught >= 1, "no pin noticed the planted mistake %r" % name
 

@@ -139,6 +139,39 @@ def test_one_softsync_with_barrier_is_synchronous_averaged_sgd(lam):
     assert rel_l2(ps32.state()[0], p.detach().numpy()) < 1e-6
 
 
+def test_hardsync_protocol_is_eq_1_and_enforces_the_barrier():
+    """Section 2.2 hardsync: theta <- theta - alpha * mean of one gradient per learner, staleness 0, and
+    nobody contributes twice or with old weights."""
+    lam, n_el, rounds = 5, 24, 12
+    a0 = float(np.float32(0.1))
+    w0 = G.normal_like(G.stream_key(15, G.STREAM_WEIGHTS), 0, n_el, 0.01).numpy()
+    ps = R.ReferencePS(n_el, lam, 1, a0, 0.0, 0.0, R.MOD_INV_STALENESS, 64)
+    ps.set_weights(w0)
+    ps.set_hardsync()
+    w = w0.astype(np.float64)
+    for r in range(rounds):
+        for l in range(lam):
+            assert ps.pull(l) == r
+        gs = [G.gradient(15, l, r, n_el, 1e-2).numpy() for l in range(lam)]
+        order = np.random.default_rng(r).permutation(lam)
+        for i, l in enumerate(order):
+            fired = ps.push(int(l), gs[l])
+            assert fired == (i == lam - 1)
+            if i == 0:
+                with pytest.raises(ValueError):
+                    ps.push(int(l), gs[l])                    # a second gradient in the same round
+        w = w - a0 * np.mean(np.stack(gs).astype(np.float64), axis=0)         # Eq. 1
+    assert rel_l2(ps.state()[0], w) < 1e-13
+    assert (ps.log()["tau"] == 0).all() and ps.timestamp == rounds
+    # a learner that did not pull the new weights is refused (its staleness would be 1)
+    for l in range(lam - 1):
+        ps.pull(l)
+    with pytest.raises(ValueError):
+        ps.push(lam - 1, gs[0])
+    with pytest.raises(ValueError):
+        R.ReferencePS(4, 4, 2, 0.1, 0.0, 0.0).set_hardsync()  # needs n = 1
+
+
 def test_downpour_case_is_per_push_sgd():
     """n = lambda with a constant rate is Downpour SGD: theta <- theta - alpha0 * dtheta per push."""
     lam, n_el, pushes = 6, 32, 120

@@ -318,3 +318,15 @@ def test_unbuilt_library_fails_loudly_but_build_module_imports(tmp_path):
     out = subprocess.run([sys.executable, "-c", code], cwd=tmp_path, capture_output=True, text=True,
                          env={**os.environ, "PYTHONPATH": str(tmp_path)})
     assert out.returncode == 0 and "loud" in out.stdout, out.stderr
+
+
+def test_plain_c_client_compiles_links_and_runs(tmp_path):
+    """The header is C (not only C++): a C99 program built with gcc drives the protocol calls."""
+    import subprocess
+    libdir = os.path.join(ROOT, "paper_1511_05950_b200")
+    exe = str(tmp_path / "c_abi_client")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                    os.path.join(ROOT, "tests", "c_abi_client.c"), "-o", exe,
+                    "-L", libdir, "-l:libsoftsync_ps.so", "-Wl,-rpath," + libdir], check=True)
+    out = subprocess.run([exe], capture_output=True, text=True)
+    assert out.returncode == 0 and "c client ok" in out.stdout, out.stdout + out.stderr

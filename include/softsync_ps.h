@@ -9,7 +9,8 @@
  *
  * Conventions
  *   - Pointers named *_dev are device pointers on the GPU that was current when
- *     ps_create ran; *_host are host pointers.  The library allocates no device
+ *     ps_create ran (later calls may be made with any device current: the library switches to
+ *     the server's GPU and back); *_host are host pointers.  The library allocates no device
  *     memory: weights, momentum and staging slots are bound by the caller.
  *   - All device work is enqueued on one stream (PS_OPT_STREAM, default: the
  *     legacy default stream).  Calls return once the work is enqueued unless

@@ -307,16 +307,13 @@ class ParameterServer:
 
     def export_state(self) -> np.ndarray:
         """Protocol state (timestamp, rate, push counts) as int64 words; weights and momentum are self.w, self.v."""
-        out = np.empty(8 + len(self._learners()), dtype=np.int64)
+        out = np.empty(8 + self.num_learners, dtype=np.int64)          # PS_STATE_WORDS(lambda)
         n = _check(ps_export_state(self._h, out.ctypes.data, out.size), "ps_export_state")
         return out[:n].copy()
 
     def import_state(self, words: np.ndarray) -> None:
         words = np.ascontiguousarray(words, dtype=np.int64)
         _check(ps_import_state(self._h, words.ctypes.data, words.size), "ps_import_state")
-
-    def _learners(self):
-        return range(self.num_learners)
 
     def kernel_time(self) -> Tuple[float, int]:
         ms, n = C.c_double(), C.c_int64()

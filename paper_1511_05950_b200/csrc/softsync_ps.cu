@@ -93,6 +93,23 @@ int cuda_fail(ps_ctx *ps, cudaError_t e)
 }
 #define PS_CUDA(ps, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail((ps), e_); } while (0)
 
+// Makes the server's GPU current for the duration of a call and restores the caller's choice afterwards,
+// so that a process driving several GPUs may call any handle at any time.
+class DeviceGuard {
+public:
+    explicit DeviceGuard(const ps_ctx *ps)
+    {
+        if (ps->device >= 0 && cudaGetDevice(&prev_) == cudaSuccess && prev_ != ps->device)
+            switched_ = cudaSetDevice(ps->device) == cudaSuccess;
+    }
+    ~DeviceGuard() { if (switched_) cudaSetDevice(prev_); }
+    DeviceGuard(const DeviceGuard &) = delete;
+    DeviceGuard &operator=(const DeviceGuard &) = delete;
+private:
+    int prev_ = -1;
+    bool switched_ = false;
+};
+
 size_t grad_elem_bytes(const ps_ctx *ps) { return ps->grad_dtype == PS_GRAD_BF16 ? 2 : 4; }
 
 int64_t ts_logical(const ps_ctx *ps) { return ps->ts_applied + static_cast<int64_t>(ps->ready.size()); }
@@ -375,6 +392,7 @@ int ps_destroy(ps_t *ps)
         std::lock_guard<std::mutex> lock(g_live_mutex);
         if (!ps || !g_live.erase(ps)) return PS_ERR_INVALID_ARG;
     }
+    DeviceGuard on_device(ps);
     if (ps->device >= 0) cudaStreamSynchronize(ps->stream);
     if (ps->copy_stream) {
         cudaStreamSynchronize(ps->copy_stream);
@@ -399,6 +417,7 @@ int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev)
 int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host)
 {
     if (!is_live(ps) || (!w_src && ps->n > 0)) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     if (ps->n > 0 && (!ps->w || !ps->v)) return PS_ERR_NO_STATE;
     const size_t bytes = static_cast<size_t>(ps->n) * sizeof(float);
     if (bytes) {
@@ -422,6 +441,7 @@ int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host)
 int ps_bind_weight_mirror(ps_t *ps, void *mirror_dev)
 {
     if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     if (reinterpret_cast<uintptr_t>(mirror_dev) & 1u) return PS_ERR_INVALID_ARG;
     if (mirror_dev && (mirror_dev == ps->w || mirror_dev == ps->v)) return PS_ERR_INVALID_ARG;
     if (!ps->ready.empty()) return PS_ERR_INVALID_ARG;               // apply or flush first
@@ -513,12 +533,14 @@ int ps_set_alpha0(ps_t *ps, float alpha0)
 int ps_apply_update(ps_t *ps)
 {
     if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     return apply_some(ps);
 }
 
 int ps_flush(ps_t *ps)
 {
     if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     int total = 0;
     while (!ps->ready.empty()) {
         const int r = apply_some(ps);
@@ -531,6 +553,7 @@ int ps_flush(ps_t *ps)
 int ps_pull_weights(ps_t *ps, float *out_dev, int64_t *ts)
 {
     if (!is_live(ps) || !ts) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     if (out_dev) {
         if (ps->n > 0 && (!ps->w || !ps->v)) return PS_ERR_NO_STATE;
         const int r = ps_flush(ps);                       // weights must belong to the returned timestamp
@@ -545,6 +568,7 @@ int ps_pull_weights(ps_t *ps, float *out_dev, int64_t *ts)
 int ps_pull_weights_bf16(ps_t *ps, void *out_dev, int64_t *ts)
 {
     if (!is_live(ps) || !ts || !out_dev) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     if (!ps->mirror || (ps->n > 0 && (!ps->w || !ps->v))) return PS_ERR_NO_STATE;
     const int r = ps_flush(ps);
     if (r < 0) return r;
@@ -557,6 +581,7 @@ int ps_pull_weights_bf16(ps_t *ps, void *out_dev, int64_t *ts)
 int ps_pull_weights_host(ps_t *ps, float *out_host, int64_t *ts)
 {
     if (!is_live(ps) || !ts || !out_host) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     if (!ps->w || !ps->v) return PS_ERR_NO_STATE;
     const int r = ps_flush(ps);
     if (r < 0) return r;
@@ -570,6 +595,7 @@ int ps_pull_weights_host(ps_t *ps, float *out_host, int64_t *ts)
 int ps_pull_weights_host_async(ps_t *ps, float *out_host, int64_t *ts)
 {
     if (!is_live(ps) || !ts || !out_host) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     if (!ps->w || !ps->v) return PS_ERR_NO_STATE;
     const int r = ps_flush(ps);
     if (r < 0) return r;
@@ -602,6 +628,7 @@ int ps_push_gradient(ps_t *ps, int learner, const void *grad_dev, int64_t ts)
 int ps_push_gradient_host(ps_t *ps, int learner, const void *grad_host, int64_t ts)
 {
     if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     const int rc = check_push(ps, learner, grad_host, ts);
     if (rc != PS_OK) return rc;
     if (!ps->staging) return PS_ERR_NO_STATE;
@@ -617,6 +644,7 @@ int ps_push_gradient_host(ps_t *ps, int learner, const void *grad_host, int64_t 
 int ps_synchronize(ps_t *ps)
 {
     if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
     if (ps->copy_stream) PS_CUDA(ps, cudaStreamSynchronize(ps->copy_stream));
     return PS_OK;
@@ -689,6 +717,7 @@ int ps_import_state(ps_t *ps, const int64_t *in_host, int64_t words)
 int ps_kernel_time(ps_t *ps, double *total_ms, int64_t *launches)
 {
     if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+    DeviceGuard on_device(ps);
     PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
     double sum = 0.0;
     for (const auto &tl : ps->timed) {

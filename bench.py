@@ -411,10 +411,12 @@ def _run_sweep(args):
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
     rng = np.random.default_rng(configs.SEED)
     points = []
-    updates, warm = 50, 5
-    for n in configs.SWEEP_SIZES:
+    updates, warm = args.sweep_updates, 5
+    sizes = [int(x) for x in args.sweep_sizes.split(",") if x] or list(configs.SWEEP_SIZES)
+    group_sizes = [int(x) for x in args.sweep_c.split(",") if x] or list(configs.SWEEP_C)
+    for n in sizes:
         for grad_dtype, tdt, gb in (("fp32", torch.float32, 4), ("bf16", torch.bfloat16, 2)):
-            for c in configs.SWEEP_C:
+            for c in group_sizes:
                 abytes = algorithmic_bytes(n, c, gb)
                 pool_n = max(c, min(64, -(-(4 * l2_bytes) // (n * gb))))
                 need = n * 8 + pool_n * n * gb + (2 << 30)
@@ -480,6 +482,9 @@ def main():
     ap.add_argument("--num-params", type=int, default=0,
                     help="run the workload's protocol on a flat vector of this many parameters (profiler captures)")
     ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over sizes, group sizes and gradient types")
+    ap.add_argument("--sweep-sizes", default="", help="comma-separated subset of the sweep's vector sizes")
+    ap.add_argument("--sweep-c", default="", help="comma-separated subset of the sweep's group sizes")
+    ap.add_argument("--sweep-updates", type=int, default=50, help="timed updates per sweep point")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     cfg = configs.BY_NAME[args.workload]

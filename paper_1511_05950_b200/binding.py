@@ -315,6 +315,10 @@ class ParameterServer:
         words = np.ascontiguousarray(words, dtype=np.int64)
         _check(ps_import_state(self._h, words.ctypes.data, words.size), "ps_import_state")
 
+    def staleness_histogram(self, first_update: int = 0) -> np.ndarray:
+        """counts[t] = gradients applied with staleness t (the quantity of Fig. 1), from the held update log."""
+        return np.bincount(self.update_log(first_update)["tau"])
+
     def kernel_time(self) -> Tuple[float, int]:
         ms, n = C.c_double(), C.c_int64()
         _check(ps_kernel_time(self._h, C.byref(ms), C.byref(n)), "ps_kernel_time")

@@ -82,6 +82,7 @@ def drive(seed, lam, n, num_params=0, device=None, steps=400):
         assert ps.timestamps()[1] == ref.timestamp
     ps.flush()
     log, rlog = ps.update_log(), ref.log()
+    assert np.array_equal(ps.staleness_histogram(), np.bincount(rlog["tau"])) if len(rlog) else True
     for f in ("update", "push_index", "ts_grad", "tau", "sigma", "learner", "position"):
         assert np.array_equal(log[f], rlog[f]), f
     assert np.array_equal(log["scale"], rlog["scale"].astype(np.float32))

@@ -91,6 +91,8 @@ int cuda_fail(ps_ctx *ps, cudaError_t e)
     ps->last_cuda_error = static_cast<int>(e);
     return PS_ERR_CUDA;
 }
+// No exception may cross the C boundary: allocation failures become PS_ERR_NOMEM.
+#define PS_CATCH_ALL catch (const std::bad_alloc &) { return PS_ERR_NOMEM; } catch (...) { return PS_ERR_INVALID_ARG; }
 #define PS_CUDA(ps, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail((ps), e_); } while (0)
 
 // Makes the server's GPU current for the duration of a call and restores the caller's choice afterwards,
@@ -354,321 +356,361 @@ extern "C" {
 int ps_create(ps_t **out, int64_t num_params, int lambda, int n,
               float alpha0, float momentum, float weight_decay, int modulation)
 {
-    if (!out) return PS_ERR_INVALID_ARG;
-    *out = nullptr;
-    if (num_params < 0 || lambda < 1 || n < 1 || n > lambda) return PS_ERR_INVALID_ARG;
-    if (modulation != PS_MOD_CONSTANT && modulation != PS_MOD_INV_STALENESS) return PS_ERR_INVALID_ARG;
-    if (lambda / n > PS_MAX_GROUP) return PS_ERR_INVALID_ARG;
-    if (!(alpha0 == alpha0) || !(momentum == momentum) || !(weight_decay == weight_decay)) return PS_ERR_INVALID_ARG;
-    ps_ctx *ps = new (std::nothrow) ps_ctx;
-    if (!ps) return PS_ERR_NOMEM;
-    ps->n = num_params; ps->lambda = lambda; ps->split = n; ps->c = lambda / n;   // Eq. 2: c = floor(lambda / n)
-    ps->alpha0 = alpha0; ps->momentum = momentum; ps->weight_decay = weight_decay;
-    ps->modulation = modulation;
-    cudaError_t e = cudaGetDevice(&ps->device);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ps->sm_count, cudaDevAttrMultiProcessorCount, ps->device);
-    if (e != cudaSuccess) {
-        // No usable GPU and there is no CPU path: only a server with zero parameters
-        // (protocol bookkeeping alone, nothing to launch) may exist without one.
-        cudaGetLastError();
-        if (num_params > 0) { delete ps; return PS_ERR_CUDA; }
-        ps->device = -1; ps->sm_count = 1;
-    }
     try {
-        ps->push_count.assign(lambda, 0);
-        ps->filling.reserve(ps->c);
-    } catch (const std::bad_alloc &) { delete ps; return PS_ERR_NOMEM; }
-    {
-        std::lock_guard<std::mutex> lock(g_live_mutex);
-        g_live.insert(ps);
-    }
-    *out = ps;
-    return PS_OK;
+        if (!out) return PS_ERR_INVALID_ARG;
+        *out = nullptr;
+        if (num_params < 0 || lambda < 1 || n < 1 || n > lambda) return PS_ERR_INVALID_ARG;
+        if (modulation != PS_MOD_CONSTANT && modulation != PS_MOD_INV_STALENESS) return PS_ERR_INVALID_ARG;
+        if (lambda / n > PS_MAX_GROUP) return PS_ERR_INVALID_ARG;
+        if (!(alpha0 == alpha0) || !(momentum == momentum) || !(weight_decay == weight_decay)) return PS_ERR_INVALID_ARG;
+        ps_ctx *ps = new (std::nothrow) ps_ctx;
+        if (!ps) return PS_ERR_NOMEM;
+        ps->n = num_params; ps->lambda = lambda; ps->split = n; ps->c = lambda / n;   // Eq. 2: c = floor(lambda / n)
+        ps->alpha0 = alpha0; ps->momentum = momentum; ps->weight_decay = weight_decay;
+        ps->modulation = modulation;
+        cudaError_t e = cudaGetDevice(&ps->device);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ps->sm_count, cudaDevAttrMultiProcessorCount, ps->device);
+        if (e != cudaSuccess) {
+            // No usable GPU and there is no CPU path: only a server with zero parameters
+            // (protocol bookkeeping alone, nothing to launch) may exist without one.
+            cudaGetLastError();
+            if (num_params > 0) { delete ps; return PS_ERR_CUDA; }
+            ps->device = -1; ps->sm_count = 1;
+        }
+        try {
+            ps->push_count.assign(lambda, 0);
+            ps->filling.reserve(ps->c);
+        } catch (const std::bad_alloc &) { delete ps; return PS_ERR_NOMEM; }
+        {
+            std::lock_guard<std::mutex> lock(g_live_mutex);
+            g_live.insert(ps);
+        }
+        *out = ps;
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_destroy(ps_t *ps)
 {
-    {
-        std::lock_guard<std::mutex> lock(g_live_mutex);
-        if (!ps || !g_live.erase(ps)) return PS_ERR_INVALID_ARG;
-    }
-    DeviceGuard on_device(ps);
-    if (ps->device >= 0) cudaStreamSynchronize(ps->stream);
-    if (ps->copy_stream) {
-        cudaStreamSynchronize(ps->copy_stream);
-        cudaEventDestroy(ps->weights_ready); cudaEventDestroy(ps->weights_copied);
-        cudaStreamDestroy(ps->copy_stream);
-    }
-    release_events(ps);
-    for (auto &tl : ps->spare_events) { cudaEventDestroy(tl.start); cudaEventDestroy(tl.stop); }
-    delete ps;
-    return PS_OK;
+    try {
+        {
+            std::lock_guard<std::mutex> lock(g_live_mutex);
+            if (!ps || !g_live.erase(ps)) return PS_ERR_INVALID_ARG;
+        }
+        DeviceGuard on_device(ps);
+        if (ps->device >= 0) cudaStreamSynchronize(ps->stream);
+        if (ps->copy_stream) {
+            cudaStreamSynchronize(ps->copy_stream);
+            cudaEventDestroy(ps->weights_ready); cudaEventDestroy(ps->weights_copied);
+            cudaStreamDestroy(ps->copy_stream);
+        }
+        release_events(ps);
+        for (auto &tl : ps->spare_events) { cudaEventDestroy(tl.start); cudaEventDestroy(tl.stop); }
+        delete ps;
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev)
 {
-    if (!is_live(ps) || !w_dev || !v_dev || w_dev == v_dev) return PS_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(w_dev) & 3u) || (reinterpret_cast<uintptr_t>(v_dev) & 3u)) return PS_ERR_INVALID_ARG;
-    if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
-    ps->w = w_dev; ps->v = v_dev;
-    return PS_OK;
+    try {
+        if (!is_live(ps) || !w_dev || !v_dev || w_dev == v_dev) return PS_ERR_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(w_dev) & 3u) || (reinterpret_cast<uintptr_t>(v_dev) & 3u)) return PS_ERR_INVALID_ARG;
+        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+        ps->w = w_dev; ps->v = v_dev;
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host)
 {
-    if (!is_live(ps) || (!w_src && ps->n > 0)) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    if (ps->n > 0 && (!ps->w || !ps->v)) return PS_ERR_NO_STATE;
-    const size_t bytes = static_cast<size_t>(ps->n) * sizeof(float);
-    if (bytes) {
-        const int rb = order_after_readback(ps);
-        if (rb != PS_OK) return rb;
-        PS_CUDA(ps, cudaMemcpyAsync(ps->w, w_src, bytes, src_is_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, ps->stream));
-        PS_CUDA(ps, cudaMemsetAsync(ps->v, 0, bytes, ps->stream));
-        const int rm = refresh_mirror(ps);
-        if (rm != PS_OK) return rm;
-        if (src_is_host) PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
-    }
-    for (auto &grp : ps->ready) for (const Entry &en : grp) if (en.slot >= 0) ps->free_slots.push_back(en.slot);
-    for (const Entry &en : ps->filling) if (en.slot >= 0) ps->free_slots.push_back(en.slot);
-    ps->ready.clear(); ps->filling.clear();
-    std::fill(ps->push_count.begin(), ps->push_count.end(), 0);
-    ps->ts_applied = 0;
-    ps->log.clear(); ps->log_first_update = 0;
-    return PS_OK;
+    try {
+        if (!is_live(ps) || (!w_src && ps->n > 0)) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        if (ps->n > 0 && (!ps->w || !ps->v)) return PS_ERR_NO_STATE;
+        const size_t bytes = static_cast<size_t>(ps->n) * sizeof(float);
+        if (bytes) {
+            const int rb = order_after_readback(ps);
+            if (rb != PS_OK) return rb;
+            PS_CUDA(ps, cudaMemcpyAsync(ps->w, w_src, bytes, src_is_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, ps->stream));
+            PS_CUDA(ps, cudaMemsetAsync(ps->v, 0, bytes, ps->stream));
+            const int rm = refresh_mirror(ps);
+            if (rm != PS_OK) return rm;
+            if (src_is_host) PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+        }
+        for (auto &grp : ps->ready) for (const Entry &en : grp) if (en.slot >= 0) ps->free_slots.push_back(en.slot);
+        for (const Entry &en : ps->filling) if (en.slot >= 0) ps->free_slots.push_back(en.slot);
+        ps->ready.clear(); ps->filling.clear();
+        std::fill(ps->push_count.begin(), ps->push_count.end(), 0);
+        ps->ts_applied = 0;
+        ps->log.clear(); ps->log_first_update = 0;
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_bind_weight_mirror(ps_t *ps, void *mirror_dev)
 {
-    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    if (reinterpret_cast<uintptr_t>(mirror_dev) & 1u) return PS_ERR_INVALID_ARG;
-    if (mirror_dev && (mirror_dev == ps->w || mirror_dev == ps->v)) return PS_ERR_INVALID_ARG;
-    if (!ps->ready.empty()) return PS_ERR_INVALID_ARG;               // apply or flush first
-    ps->mirror = static_cast<unsigned short *>(mirror_dev);
-    return refresh_mirror(ps);
+    try {
+        if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        if (reinterpret_cast<uintptr_t>(mirror_dev) & 1u) return PS_ERR_INVALID_ARG;
+        if (mirror_dev && (mirror_dev == ps->w || mirror_dev == ps->v)) return PS_ERR_INVALID_ARG;
+        if (!ps->ready.empty()) return PS_ERR_INVALID_ARG;               // apply or flush first
+        ps->mirror = static_cast<unsigned short *>(mirror_dev);
+        return refresh_mirror(ps);
+    } PS_CATCH_ALL
 }
 
 int ps_bind_staging(ps_t *ps, void *slots_dev, int64_t slot_bytes, int num_slots)
 {
-    if (!is_live(ps) || !slots_dev || num_slots < 1 || slot_bytes < 0) return PS_ERR_INVALID_ARG;
-    if (!aligned16(slots_dev) || (slot_bytes & 15)) return PS_ERR_INVALID_ARG;
-    if (slot_bytes < ps->n * static_cast<int64_t>(grad_elem_bytes(ps))) return PS_ERR_INVALID_ARG;
-    if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
-    ps->staging = static_cast<char *>(slots_dev);
-    ps->slot_bytes = slot_bytes; ps->num_slots = num_slots;
-    ps->free_slots.clear();
-    for (int s = num_slots - 1; s >= 0; --s) ps->free_slots.push_back(s);
-    return PS_OK;
+    try {
+        if (!is_live(ps) || !slots_dev || num_slots < 1 || slot_bytes < 0) return PS_ERR_INVALID_ARG;
+        if (!aligned16(slots_dev) || (slot_bytes & 15)) return PS_ERR_INVALID_ARG;
+        if (slot_bytes < ps->n * static_cast<int64_t>(grad_elem_bytes(ps))) return PS_ERR_INVALID_ARG;
+        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+        ps->staging = static_cast<char *>(slots_dev);
+        ps->slot_bytes = slot_bytes; ps->num_slots = num_slots;
+        ps->free_slots.clear();
+        for (int s = num_slots - 1; s >= 0; --s) ps->free_slots.push_back(s);
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_set_option(ps_t *ps, int key, int64_t value)
 {
-    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
-    switch (key) {
-    case PS_OPT_GRAD_DTYPE:
-        if (value != PS_GRAD_FP32 && value != PS_GRAD_BF16) return PS_ERR_INVALID_ARG;
-        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
-        if (ps->staging && ps->slot_bytes < ps->n * (value == PS_GRAD_BF16 ? 2 : 4)) return PS_ERR_INVALID_ARG;
-        ps->grad_dtype = static_cast<int>(value); return PS_OK;
-    case PS_OPT_FUSE_T:
-        if (value < 1 || value > PS_MAX_FUSE_T) return PS_ERR_INVALID_ARG;
-        ps->fuse_t = static_cast<int>(value); return PS_OK;
-    case PS_OPT_STREAM:
-        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
-        ps->stream = reinterpret_cast<cudaStream_t>(static_cast<uintptr_t>(value)); return PS_OK;
-    case PS_OPT_QUEUE_GROUPS:
-        if (value < 1) return PS_ERR_INVALID_ARG;
-        ps->queue_groups = value; return PS_OK;
-    case PS_OPT_LOG_UPDATES:
-        if (value < 0) return PS_ERR_INVALID_ARG;
-        ps->log_updates = value; return PS_OK;
-    case PS_OPT_TIMING:
-        if (value != 0 && value != 1) return PS_ERR_INVALID_ARG;
-        ps->timing = static_cast<int>(value); return PS_OK;
-    case PS_OPT_KERNEL:
-        if (value < PS_KERNEL_AUTO || value > PS_KERNEL_VECTOR) return PS_ERR_INVALID_ARG;
-        ps->kernel_choice = static_cast<int>(value); return PS_OK;
-    case PS_OPT_PROTOCOL:
-        if (value != PS_PROTOCOL_SOFTSYNC && value != PS_PROTOCOL_HARDSYNC) return PS_ERR_INVALID_ARG;
-        if (value == PS_PROTOCOL_HARDSYNC && ps->split != 1) return PS_ERR_INVALID_ARG;
-        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
-        ps->protocol = static_cast<int>(value); return PS_OK;
-    case PS_OPT_OVERLAP_LAUNCH:
-        if (value != 0 && value != 1) return PS_ERR_INVALID_ARG;
-        ps->overlap_launch = static_cast<int>(value); return PS_OK;
-    case PS_OPT_BLOCK_THREADS:
-        if (value != 0 && value != 128 && value != 256 && value != 512) return PS_ERR_INVALID_ARG;
-        ps->block_threads = static_cast<int>(value); return PS_OK;
-    default:
-        return PS_ERR_INVALID_ARG;
-    }
+    try {
+        if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+        switch (key) {
+        case PS_OPT_GRAD_DTYPE:
+            if (value != PS_GRAD_FP32 && value != PS_GRAD_BF16) return PS_ERR_INVALID_ARG;
+            if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+            if (ps->staging && ps->slot_bytes < ps->n * (value == PS_GRAD_BF16 ? 2 : 4)) return PS_ERR_INVALID_ARG;
+            ps->grad_dtype = static_cast<int>(value); return PS_OK;
+        case PS_OPT_FUSE_T:
+            if (value < 1 || value > PS_MAX_FUSE_T) return PS_ERR_INVALID_ARG;
+            ps->fuse_t = static_cast<int>(value); return PS_OK;
+        case PS_OPT_STREAM:
+            if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+            ps->stream = reinterpret_cast<cudaStream_t>(static_cast<uintptr_t>(value)); return PS_OK;
+        case PS_OPT_QUEUE_GROUPS:
+            if (value < 1) return PS_ERR_INVALID_ARG;
+            ps->queue_groups = value; return PS_OK;
+        case PS_OPT_LOG_UPDATES:
+            if (value < 0) return PS_ERR_INVALID_ARG;
+            ps->log_updates = value; return PS_OK;
+        case PS_OPT_TIMING:
+            if (value != 0 && value != 1) return PS_ERR_INVALID_ARG;
+            ps->timing = static_cast<int>(value); return PS_OK;
+        case PS_OPT_KERNEL:
+            if (value < PS_KERNEL_AUTO || value > PS_KERNEL_VECTOR) return PS_ERR_INVALID_ARG;
+            ps->kernel_choice = static_cast<int>(value); return PS_OK;
+        case PS_OPT_PROTOCOL:
+            if (value != PS_PROTOCOL_SOFTSYNC && value != PS_PROTOCOL_HARDSYNC) return PS_ERR_INVALID_ARG;
+            if (value == PS_PROTOCOL_HARDSYNC && ps->split != 1) return PS_ERR_INVALID_ARG;
+            if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+            ps->protocol = static_cast<int>(value); return PS_OK;
+        case PS_OPT_OVERLAP_LAUNCH:
+            if (value != 0 && value != 1) return PS_ERR_INVALID_ARG;
+            ps->overlap_launch = static_cast<int>(value); return PS_OK;
+        case PS_OPT_BLOCK_THREADS:
+            if (value != 0 && value != 128 && value != 256 && value != 512) return PS_ERR_INVALID_ARG;
+            ps->block_threads = static_cast<int>(value); return PS_OK;
+        default:
+            return PS_ERR_INVALID_ARG;
+        }
+    } PS_CATCH_ALL
 }
 
 int ps_get_option(ps_t *ps, int key, int64_t *value)
 {
-    if (!is_live(ps) || !value) return PS_ERR_INVALID_ARG;
-    switch (key) {
-    case PS_OPT_GRAD_DTYPE: *value = ps->grad_dtype; return PS_OK;
-    case PS_OPT_FUSE_T: *value = ps->fuse_t; return PS_OK;
-    case PS_OPT_STREAM: *value = static_cast<int64_t>(reinterpret_cast<uintptr_t>(ps->stream)); return PS_OK;
-    case PS_OPT_QUEUE_GROUPS: *value = ps->queue_groups; return PS_OK;
-    case PS_OPT_LOG_UPDATES: *value = ps->log_updates; return PS_OK;
-    case PS_OPT_TIMING: *value = ps->timing; return PS_OK;
-    case PS_OPT_KERNEL: *value = ps->kernel_choice; return PS_OK;
-    case PS_OPT_BLOCK_THREADS: *value = ps->block_threads; return PS_OK;
-    case PS_OPT_OVERLAP_LAUNCH: *value = ps->overlap_launch; return PS_OK;
-    case PS_OPT_PROTOCOL: *value = ps->protocol; return PS_OK;
-    default: return PS_ERR_INVALID_ARG;
-    }
+    try {
+        if (!is_live(ps) || !value) return PS_ERR_INVALID_ARG;
+        switch (key) {
+        case PS_OPT_GRAD_DTYPE: *value = ps->grad_dtype; return PS_OK;
+        case PS_OPT_FUSE_T: *value = ps->fuse_t; return PS_OK;
+        case PS_OPT_STREAM: *value = static_cast<int64_t>(reinterpret_cast<uintptr_t>(ps->stream)); return PS_OK;
+        case PS_OPT_QUEUE_GROUPS: *value = ps->queue_groups; return PS_OK;
+        case PS_OPT_LOG_UPDATES: *value = ps->log_updates; return PS_OK;
+        case PS_OPT_TIMING: *value = ps->timing; return PS_OK;
+        case PS_OPT_KERNEL: *value = ps->kernel_choice; return PS_OK;
+        case PS_OPT_BLOCK_THREADS: *value = ps->block_threads; return PS_OK;
+        case PS_OPT_OVERLAP_LAUNCH: *value = ps->overlap_launch; return PS_OK;
+        case PS_OPT_PROTOCOL: *value = ps->protocol; return PS_OK;
+        default: return PS_ERR_INVALID_ARG;
+        }
+    } PS_CATCH_ALL
 }
 
 int ps_set_alpha0(ps_t *ps, float alpha0)
 {
-    if (!is_live(ps) || !(alpha0 == alpha0)) return PS_ERR_INVALID_ARG;
-    ps->alpha0 = alpha0;
-    return PS_OK;
+    try {
+        if (!is_live(ps) || !(alpha0 == alpha0)) return PS_ERR_INVALID_ARG;
+        ps->alpha0 = alpha0;
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_apply_update(ps_t *ps)
 {
-    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    return apply_some(ps);
+    try {
+        if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        return apply_some(ps);
+    } PS_CATCH_ALL
 }
 
 int ps_flush(ps_t *ps)
 {
-    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    int total = 0;
-    while (!ps->ready.empty()) {
-        const int r = apply_some(ps);
-        if (r < 0) return r;
-        total += r;
-    }
-    return total;
+    try {
+        if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        int total = 0;
+        while (!ps->ready.empty()) {
+            const int r = apply_some(ps);
+            if (r < 0) return r;
+            total += r;
+        }
+        return total;
+    } PS_CATCH_ALL
 }
 
 int ps_pull_weights(ps_t *ps, float *out_dev, int64_t *ts)
 {
-    if (!is_live(ps) || !ts) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    if (out_dev) {
-        if (ps->n > 0 && (!ps->w || !ps->v)) return PS_ERR_NO_STATE;
-        const int r = ps_flush(ps);                       // weights must belong to the returned timestamp
-        if (r < 0) return r;
-        if (ps->n) PS_CUDA(ps, cudaMemcpyAsync(out_dev, ps->w, static_cast<size_t>(ps->n) * sizeof(float),
-                                               cudaMemcpyDeviceToDevice, ps->stream));
-    }
-    *ts = ts_logical(ps);
-    return PS_OK;
+    try {
+        if (!is_live(ps) || !ts) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        if (out_dev) {
+            if (ps->n > 0 && (!ps->w || !ps->v)) return PS_ERR_NO_STATE;
+            const int r = ps_flush(ps);                       // weights must belong to the returned timestamp
+            if (r < 0) return r;
+            if (ps->n) PS_CUDA(ps, cudaMemcpyAsync(out_dev, ps->w, static_cast<size_t>(ps->n) * sizeof(float),
+                                                   cudaMemcpyDeviceToDevice, ps->stream));
+        }
+        *ts = ts_logical(ps);
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_pull_weights_bf16(ps_t *ps, void *out_dev, int64_t *ts)
 {
-    if (!is_live(ps) || !ts || !out_dev) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    if (!ps->mirror || (ps->n > 0 && (!ps->w || !ps->v))) return PS_ERR_NO_STATE;
-    const int r = ps_flush(ps);
-    if (r < 0) return r;
-    if (ps->n) PS_CUDA(ps, cudaMemcpyAsync(out_dev, ps->mirror, static_cast<size_t>(ps->n) * 2,
-                                           cudaMemcpyDeviceToDevice, ps->stream));
-    *ts = ts_logical(ps);
-    return PS_OK;
+    try {
+        if (!is_live(ps) || !ts || !out_dev) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        if (!ps->mirror || (ps->n > 0 && (!ps->w || !ps->v))) return PS_ERR_NO_STATE;
+        const int r = ps_flush(ps);
+        if (r < 0) return r;
+        if (ps->n) PS_CUDA(ps, cudaMemcpyAsync(out_dev, ps->mirror, static_cast<size_t>(ps->n) * 2,
+                                               cudaMemcpyDeviceToDevice, ps->stream));
+        *ts = ts_logical(ps);
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_pull_weights_host(ps_t *ps, float *out_host, int64_t *ts)
 {
-    if (!is_live(ps) || !ts || !out_host) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    if (!ps->w || !ps->v) return PS_ERR_NO_STATE;
-    const int r = ps_flush(ps);
-    if (r < 0) return r;
-    if (ps->n) PS_CUDA(ps, cudaMemcpyAsync(out_host, ps->w, static_cast<size_t>(ps->n) * sizeof(float),
-                                           cudaMemcpyDeviceToHost, ps->stream));
-    PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
-    *ts = ts_logical(ps);
-    return PS_OK;
+    try {
+        if (!is_live(ps) || !ts || !out_host) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        if (!ps->w || !ps->v) return PS_ERR_NO_STATE;
+        const int r = ps_flush(ps);
+        if (r < 0) return r;
+        if (ps->n) PS_CUDA(ps, cudaMemcpyAsync(out_host, ps->w, static_cast<size_t>(ps->n) * sizeof(float),
+                                               cudaMemcpyDeviceToHost, ps->stream));
+        PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+        *ts = ts_logical(ps);
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_pull_weights_host_async(ps_t *ps, float *out_host, int64_t *ts)
 {
-    if (!is_live(ps) || !ts || !out_host) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    if (!ps->w || !ps->v) return PS_ERR_NO_STATE;
-    const int r = ps_flush(ps);
-    if (r < 0) return r;
-    if (!ps->copy_stream) {
-        PS_CUDA(ps, cudaStreamCreateWithFlags(&ps->copy_stream, cudaStreamNonBlocking));
-        PS_CUDA(ps, cudaEventCreateWithFlags(&ps->weights_ready, cudaEventDisableTiming));
-        PS_CUDA(ps, cudaEventCreateWithFlags(&ps->weights_copied, cudaEventDisableTiming));
-    }
-    if (ps->n) {
-        PS_CUDA(ps, cudaEventRecord(ps->weights_ready, ps->stream));
-        PS_CUDA(ps, cudaStreamWaitEvent(ps->copy_stream, ps->weights_ready, 0));
-        PS_CUDA(ps, cudaMemcpyAsync(out_host, ps->w, static_cast<size_t>(ps->n) * sizeof(float),
-                                    cudaMemcpyDeviceToHost, ps->copy_stream));
-        PS_CUDA(ps, cudaEventRecord(ps->weights_copied, ps->copy_stream));
-        ps->copy_in_flight = true;
-    }
-    *ts = ts_logical(ps);
-    return PS_OK;
+    try {
+        if (!is_live(ps) || !ts || !out_host) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        if (!ps->w || !ps->v) return PS_ERR_NO_STATE;
+        const int r = ps_flush(ps);
+        if (r < 0) return r;
+        if (!ps->copy_stream) {
+            PS_CUDA(ps, cudaStreamCreateWithFlags(&ps->copy_stream, cudaStreamNonBlocking));
+            PS_CUDA(ps, cudaEventCreateWithFlags(&ps->weights_ready, cudaEventDisableTiming));
+            PS_CUDA(ps, cudaEventCreateWithFlags(&ps->weights_copied, cudaEventDisableTiming));
+        }
+        if (ps->n) {
+            PS_CUDA(ps, cudaEventRecord(ps->weights_ready, ps->stream));
+            PS_CUDA(ps, cudaStreamWaitEvent(ps->copy_stream, ps->weights_ready, 0));
+            PS_CUDA(ps, cudaMemcpyAsync(out_host, ps->w, static_cast<size_t>(ps->n) * sizeof(float),
+                                        cudaMemcpyDeviceToHost, ps->copy_stream));
+            PS_CUDA(ps, cudaEventRecord(ps->weights_copied, ps->copy_stream));
+            ps->copy_in_flight = true;
+        }
+        *ts = ts_logical(ps);
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_push_gradient(ps_t *ps, int learner, const void *grad_dev, int64_t ts)
 {
-    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
-    const int rc = check_push(ps, learner, grad_dev, ts);
-    if (rc != PS_OK) return rc;
-    if (reinterpret_cast<uintptr_t>(grad_dev) & (grad_elem_bytes(ps) - 1)) return PS_ERR_INVALID_ARG;
-    return push_common(ps, learner, grad_dev, ts, -1);
+    try {
+        if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+        const int rc = check_push(ps, learner, grad_dev, ts);
+        if (rc != PS_OK) return rc;
+        if (reinterpret_cast<uintptr_t>(grad_dev) & (grad_elem_bytes(ps) - 1)) return PS_ERR_INVALID_ARG;
+        return push_common(ps, learner, grad_dev, ts, -1);
+    } PS_CATCH_ALL
 }
 
 int ps_push_gradient_host(ps_t *ps, int learner, const void *grad_host, int64_t ts)
 {
-    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    const int rc = check_push(ps, learner, grad_host, ts);
-    if (rc != PS_OK) return rc;
-    if (!ps->staging) return PS_ERR_NO_STATE;
-    if (ps->free_slots.empty()) return PS_ERR_QUEUE_FULL;
-    const int slot = ps->free_slots.back();
-    char *dst = ps->staging + static_cast<int64_t>(slot) * ps->slot_bytes;
-    const size_t bytes = static_cast<size_t>(ps->n) * grad_elem_bytes(ps);
-    if (bytes) PS_CUDA(ps, cudaMemcpyAsync(dst, grad_host, bytes, cudaMemcpyHostToDevice, ps->stream));
-    ps->free_slots.pop_back();
-    return push_common(ps, learner, dst, ts, slot);
+    try {
+        if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        const int rc = check_push(ps, learner, grad_host, ts);
+        if (rc != PS_OK) return rc;
+        if (!ps->staging) return PS_ERR_NO_STATE;
+        if (ps->free_slots.empty()) return PS_ERR_QUEUE_FULL;
+        const int slot = ps->free_slots.back();
+        char *dst = ps->staging + static_cast<int64_t>(slot) * ps->slot_bytes;
+        const size_t bytes = static_cast<size_t>(ps->n) * grad_elem_bytes(ps);
+        if (bytes) PS_CUDA(ps, cudaMemcpyAsync(dst, grad_host, bytes, cudaMemcpyHostToDevice, ps->stream));
+        ps->free_slots.pop_back();
+        return push_common(ps, learner, dst, ts, slot);
+    } PS_CATCH_ALL
 }
 
 int ps_synchronize(ps_t *ps)
 {
-    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
-    if (ps->copy_stream) PS_CUDA(ps, cudaStreamSynchronize(ps->copy_stream));
-    return PS_OK;
+    try {
+        if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+        if (ps->copy_stream) PS_CUDA(ps, cudaStreamSynchronize(ps->copy_stream));
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_get_update_log(ps_t *ps, int64_t first_update, int64_t count, ps_log_entry *out_host)
 {
-    if (!is_live(ps) || count < 0 || (count > 0 && !out_host)) return PS_ERR_INVALID_ARG;
-    const int64_t held = static_cast<int64_t>(ps->log.size()) / ps->c;
-    if (first_update < ps->log_first_update || first_update + count > ps->log_first_update + held)
-        return PS_ERR_LOG_EVICTED;
-    const int64_t off = (first_update - ps->log_first_update) * ps->c;
-    std::copy(ps->log.begin() + off, ps->log.begin() + off + count * ps->c, out_host);
-    return PS_OK;
+    try {
+        if (!is_live(ps) || count < 0 || (count > 0 && !out_host)) return PS_ERR_INVALID_ARG;
+        const int64_t held = static_cast<int64_t>(ps->log.size()) / ps->c;
+        if (first_update < ps->log_first_update || first_update + count > ps->log_first_update + held)
+            return PS_ERR_LOG_EVICTED;
+        const int64_t off = (first_update - ps->log_first_update) * ps->c;
+        std::copy(ps->log.begin() + off, ps->log.begin() + off + count * ps->c, out_host);
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_peek_state(ps_t *ps, const float **w_dev, const float **v_dev, int64_t *ts_applied, int64_t *ts_log)
 {
-    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
-    if (w_dev) *w_dev = ps->w;
-    if (v_dev) *v_dev = ps->v;
-    if (ts_applied) *ts_applied = ps->ts_applied;
-    if (ts_log) *ts_log = ts_logical(ps);
-    return PS_OK;
+    try {
+        if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+        if (w_dev) *w_dev = ps->w;
+        if (v_dev) *v_dev = ps->v;
+        if (ts_applied) *ts_applied = ps->ts_applied;
+        if (ts_log) *ts_log = ts_logical(ps);
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 namespace {
@@ -679,56 +721,62 @@ constexpr int64_t kStateHeader = 8;
 
 int ps_export_state(ps_t *ps, int64_t *out_host, int64_t capacity_words)
 {
-    if (!is_live(ps) || !out_host) return PS_ERR_INVALID_ARG;
-    const int64_t words = kStateHeader + ps->lambda;
-    if (capacity_words < words) return PS_ERR_INVALID_ARG;
-    if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_NOT_READY;   // borrowed gradients cannot be saved
-    uint32_t alpha_bits;
-    static_assert(sizeof alpha_bits == sizeof ps->alpha0, "fp32 rate");
-    std::memcpy(&alpha_bits, &ps->alpha0, sizeof alpha_bits);
-    out_host[0] = kStateMagic; out_host[1] = kStateVersion;
-    out_host[2] = ps->n; out_host[3] = ps->lambda; out_host[4] = ps->split;
-    out_host[5] = ps->ts_applied; out_host[6] = static_cast<int64_t>(alpha_bits); out_host[7] = ps->launches;
-    for (int l = 0; l < ps->lambda; ++l) out_host[kStateHeader + l] = ps->push_count[l];
-    return static_cast<int>(words);
+    try {
+        if (!is_live(ps) || !out_host) return PS_ERR_INVALID_ARG;
+        const int64_t words = kStateHeader + ps->lambda;
+        if (capacity_words < words) return PS_ERR_INVALID_ARG;
+        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_NOT_READY;   // borrowed gradients cannot be saved
+        uint32_t alpha_bits;
+        static_assert(sizeof alpha_bits == sizeof ps->alpha0, "fp32 rate");
+        std::memcpy(&alpha_bits, &ps->alpha0, sizeof alpha_bits);
+        out_host[0] = kStateMagic; out_host[1] = kStateVersion;
+        out_host[2] = ps->n; out_host[3] = ps->lambda; out_host[4] = ps->split;
+        out_host[5] = ps->ts_applied; out_host[6] = static_cast<int64_t>(alpha_bits); out_host[7] = ps->launches;
+        for (int l = 0; l < ps->lambda; ++l) out_host[kStateHeader + l] = ps->push_count[l];
+        return static_cast<int>(words);
+    } PS_CATCH_ALL
 }
 
 int ps_import_state(ps_t *ps, const int64_t *in_host, int64_t words)
 {
-    if (!is_live(ps) || !in_host || words < kStateHeader) return PS_ERR_INVALID_ARG;
-    if (in_host[0] != kStateMagic || in_host[1] != kStateVersion) return PS_ERR_INVALID_ARG;
-    if (in_host[2] != ps->n || in_host[3] != ps->lambda || in_host[4] != ps->split) return PS_ERR_INVALID_ARG;
-    if (words != kStateHeader + ps->lambda || in_host[5] < 0 || in_host[7] < 0) return PS_ERR_INVALID_ARG;
-    for (int l = 0; l < ps->lambda; ++l) if (in_host[kStateHeader + l] < 0) return PS_ERR_INVALID_ARG;
-    if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_NOT_READY;
-    const uint32_t alpha_bits = static_cast<uint32_t>(in_host[6]);
-    float alpha0;
-    std::memcpy(&alpha0, &alpha_bits, sizeof alpha0);
-    if (!(alpha0 == alpha0)) return PS_ERR_INVALID_ARG;
-    ps->alpha0 = alpha0;
-    ps->ts_applied = in_host[5];
-    ps->launches = in_host[7];
-    for (int l = 0; l < ps->lambda; ++l) ps->push_count[l] = in_host[kStateHeader + l];
-    ps->log.clear();
-    ps->log_first_update = ps->ts_applied;
-    return PS_OK;
+    try {
+        if (!is_live(ps) || !in_host || words < kStateHeader) return PS_ERR_INVALID_ARG;
+        if (in_host[0] != kStateMagic || in_host[1] != kStateVersion) return PS_ERR_INVALID_ARG;
+        if (in_host[2] != ps->n || in_host[3] != ps->lambda || in_host[4] != ps->split) return PS_ERR_INVALID_ARG;
+        if (words != kStateHeader + ps->lambda || in_host[5] < 0 || in_host[7] < 0) return PS_ERR_INVALID_ARG;
+        for (int l = 0; l < ps->lambda; ++l) if (in_host[kStateHeader + l] < 0) return PS_ERR_INVALID_ARG;
+        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_NOT_READY;
+        const uint32_t alpha_bits = static_cast<uint32_t>(in_host[6]);
+        float alpha0;
+        std::memcpy(&alpha0, &alpha_bits, sizeof alpha0);
+        if (!(alpha0 == alpha0)) return PS_ERR_INVALID_ARG;
+        ps->alpha0 = alpha0;
+        ps->ts_applied = in_host[5];
+        ps->launches = in_host[7];
+        for (int l = 0; l < ps->lambda; ++l) ps->push_count[l] = in_host[kStateHeader + l];
+        ps->log.clear();
+        ps->log_first_update = ps->ts_applied;
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_kernel_time(ps_t *ps, double *total_ms, int64_t *launches)
 {
-    if (!is_live(ps)) return PS_ERR_INVALID_ARG;
-    DeviceGuard on_device(ps);
-    PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
-    double sum = 0.0;
-    for (const auto &tl : ps->timed) {
-        float ms = 0.f;
-        PS_CUDA(ps, cudaEventElapsedTime(&ms, tl.start, tl.stop));
-        sum += ms;
-    }
-    if (total_ms) *total_ms = sum;
-    if (launches) *launches = static_cast<int64_t>(ps->timed.size());
-    release_events(ps);
-    return PS_OK;
+    try {
+        if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+        double sum = 0.0;
+        for (const auto &tl : ps->timed) {
+            float ms = 0.f;
+            PS_CUDA(ps, cudaEventElapsedTime(&ms, tl.start, tl.stop));
+            sum += ms;
+        }
+        if (total_ms) *total_ms = sum;
+        if (launches) *launches = static_cast<int64_t>(ps->timed.size());
+        release_events(ps);
+        return PS_OK;
+    } PS_CATCH_ALL
 }
 
 int ps_last_cuda_error(ps_t *ps)

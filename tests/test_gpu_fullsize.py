@@ -96,6 +96,9 @@ def run_full(cfg, lazy, num_pushes=None, overlap=False):
     w64, v64 = refs[64].state()
     tol = 1e-3 if cfg.grad_dtype == "bf16" else 1e-5
     assert rel_l2(w, w64) <= tol and rel_l2(v, v64) <= tol
+    run_full.last_stats = {"gpu_vs_fp64_w": rel_l2(w, w64), "gpu_vs_fp64_v": rel_l2(v, v64),
+                           "fp32ref_vs_fp64_w": rel_l2(w32, w64), "fp32ref_vs_fp64_v": rel_l2(v32, v64),
+                           "sampled_elements": int(idx.numel()), "updates": int(pushes // cfg.c)}
     return log
 
 

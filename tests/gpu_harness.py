@@ -39,7 +39,7 @@ def replay_gpu(ps: P.ParameterServer, kinds, learners, grad_fn, lazy: bool = Fal
 
 def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, grad_std, kinds, learners,
              w0: torch.Tensor, seed: int, fuse_t: int = 1, lazy: bool = False, precisions=(32, 64),
-             options=None, misalign: int = 0):
+             options=None, misalign: int = 0, checkpoints: int = 0, tol: float = 1e-5):
     """Returns (gpu_w, gpu_v, gpu_log, {precision: (w, v, log)})."""
     dev = torch.device("cuda", 0)
     tdt = TORCH_DTYPE[grad_dtype]
@@ -76,6 +76,9 @@ def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, g
     # the reference consumes pulls too: interleave by wrapping the replay
     pulled, counts = {}, {}
     ready = 0
+    total_updates = int((kinds != PULL).sum()) // (lam // n)
+    every = max(1, total_updates // checkpoints) if checkpoints else 0
+    next_check = every
     for k, l in zip(kinds.tolist(), learners.tolist()):
         if k == PULL:
             pulled[l] = ps.pull_weights()
@@ -87,6 +90,18 @@ def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, g
             ready += ps.push_gradient(l, grad_fn(l, p), pulled[l])
             if ready and (not lazy or ready >= fuse_t):
                 ready -= ps.apply_update()
+            applied = ps.timestamps()[0]
+            if every and ready == 0 and applied >= next_check:       # intermediate states, not only the final one
+                next_check = applied + every
+                ps.synchronize()
+                wc, vc = ps.w[:num_params].cpu().numpy(), ps.v[:num_params].cpu().numpy()
+                for prec, r in refs.items():
+                    assert r.timestamp == applied
+                    wr, vr = r.state()
+                    if prec == 32:
+                        assert np.array_equal(wc, wr.astype(np.float32)) and np.array_equal(vc, vr.astype(np.float32))
+                    else:
+                        assert rel_l2(wc, wr) <= tol and rel_l2(vc, vr) <= tol
     ps.flush()
     ps.synchronize()
     out = {prec: (*r.state(), r.log()) for prec, r in refs.items()}

@@ -34,16 +34,16 @@ def run_config(cfg, num_pushes=None, layout=None, **kw):
 
 
 def test_tiny_softsync_full():
-    """Config 1 in full: lambda=4, n=1, 89,578 elements, 200 updates."""
+    """Config 1 in full: lambda=4, n=1, 89,578 elements, 200 updates; state compared at every tenth of the run."""
     cfg = configs.TINY_SOFTSYNC
-    worst, log = run_config(cfg)
+    worst, log = run_config(cfg, checkpoints=10)
     assert log["update"][-1] == 199 and (log["sigma"] == 1).all()
 
 
 def test_pure_async_full():
     """Config 2 in full: lambda=30, n=30, 10,000 pushes with Exp(1) compute times."""
     cfg = configs.PURE_ASYNC
-    worst, log = run_config(cfg)
+    worst, log = run_config(cfg, checkpoints=10)
     assert len(log) == 10000 and log["sigma"].max() > 60
 
 

@@ -408,6 +408,44 @@ def test_hardsync_protocol_matches_reference():
     assert (log["tau"] == 0).all()
 
 
+def test_two_servers_on_their_own_streams():
+    """Each server enqueues on the stream it was given; two servers on two streams run concurrently
+    and independently, and each matches the reference."""
+    from tests.gpu_harness import as_reference_grad
+    dev = torch.device("cuda", 0)
+    n_el, lam = 600011, 3
+    streams = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    servers, refs, grads = [], [], []
+    w0 = G.initial_weights(layouts.flat(n_el), 31)
+    for k, st in enumerate(streams):
+        with torch.cuda.stream(st):
+            ps = P.ParameterServer(n_el, lam, 1, 0.01 * (k + 1), 0.9, 5e-4, device=dev)
+            assert ps.get_option(P.PS_OPT_STREAM) == st.cuda_stream
+            ps.init_weights(w0.to(dev))
+            gs = [[G.gradient(31 + k, l, u, n_el, 1e-3, device=dev) for l in range(lam)] for u in range(6)]
+        ref = R.ReferencePS(n_el, lam, 1, 0.01 * (k + 1), 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+        ref.set_weights(w0.numpy())
+        servers.append(ps); refs.append(ref); grads.append(gs)
+    torch.cuda.synchronize()
+    for u in range(6):                                   # interleave the two servers' launches
+        for k, st in enumerate(streams):
+            with torch.cuda.stream(st):
+                ts = servers[k].pull_weights()
+                for l in range(lam):
+                    servers[k].push_gradient(l, grads[k][u][l], ts)
+                assert servers[k].apply_update() == 1
+    for k, st in enumerate(streams):
+        for u in range(6):
+            for l in range(lam):
+                refs[k].pull(l)
+            for l in range(lam):
+                refs[k].push(l, as_reference_grad(grads[k][u][l]))
+        servers[k].synchronize()
+        assert np.array_equal(servers[k].w.cpu().numpy(), refs[k].state()[0].astype(np.float32))
+        assert np.array_equal(servers[k].v.cpu().numpy(), refs[k].state()[1].astype(np.float32))
+        servers[k].destroy()
+
+
 def test_zero_parameters():
     _simple(0, 4, 2, 12)
 

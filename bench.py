@@ -260,15 +260,19 @@ def run_ours(args, cfg, rank, world, local_rank):
     elapsed_ms, e2e_ms, kern_ms = max_over_ranks([elapsed_ms, e2e_s * 1e3, kernel_ms / max(1, launches)], dev, world)
 
     elems_per_step = cfg.c * n * groups_per_step
-    value = whole_job_value(world, elems_per_step, args.steps, elapsed_ms)
-    e2e_value = whole_job_value(world, elems_per_step, e2e_steps, e2e_ms) if e2e_steps else None
+    if args.total_params:                              # sharded: the ranks together hold one vector
+        value = whole_job_value(1, cfg.c * args.total_params * groups_per_step, args.steps, elapsed_ms)
+        e2e_value = whole_job_value(1, cfg.c * args.total_params * groups_per_step, e2e_steps, e2e_ms) if e2e_steps else None
+    else:
+        value = whole_job_value(world, elems_per_step, args.steps, elapsed_ms)
+        e2e_value = whole_job_value(world, elems_per_step, e2e_steps, e2e_ms) if e2e_steps else None
     abytes = algorithmic_bytes(n, cfg.c * fuse_t, gbytes) + (2 * n if args.bf16_mirror else 0)
     peak, peak_kind = hbm_peak()
     achieved = abytes / (kern_ms * 1e-3) / 1e9
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "strong" if args.total_params else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {
             "workload": "%s: N=%d fp32 parameters (AlexNet-like layout), lambda=%d, n=%d, c=%d %s gradients "
                         "per update, T=%d updates per kernel pass" % (cfg.name, n, cfg.num_learners, cfg.n, cfg.c,
@@ -278,7 +282,9 @@ def run_ours(args, cfg, rank, world, local_rank):
             "momentum": cfg.momentum, "weight_decay": cfg.weight_decay, "modulation": cfg.modulation,
             "bf16_mirror": bool(args.bf16_mirror),
             "launch": "ordinary" if args.no_overlap else "programmatic dependent launch (PS_OPT_OVERLAP_LAUNCH=1)",
-            "parallelism": "replicas only (independent servers, no data-path collective)" if world > 1 else "1 GPU",
+            "parallelism": ("%d contiguous shards of one %d-parameter vector, no data-path collective"
+                            % (world, args.total_params)) if args.total_params else
+                           ("replicas only (independent servers, no data-path collective)" if world > 1 else "1 GPU"),
             "l2": ("inputs larger than L2: each step streams %.2f GB from %d rotating gradient buffers"
                    % (abytes / 1e9, pool_n)) if abytes > 2 * L2_BYTES else
                   ("working set of %.1f MB per step stays in L2: a launch-latency figure, not an HBM one"
@@ -481,6 +487,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
     ap.add_argument("--num-params", type=int, default=0,
                     help="run the workload's protocol on a flat vector of this many parameters (profiler captures)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="with N > 1 ranks: one server over the workload's vector, a contiguous shard per rank "
+                         "(strong scaling) instead of one replica per rank")
     ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over sizes, group sizes and gradient types")
     ap.add_argument("--sweep-sizes", default="", help="comma-separated subset of the sweep's vector sizes")
     ap.add_argument("--sweep-c", default="", help="comma-separated subset of the sweep's group sizes")
@@ -502,6 +511,15 @@ def main():
         if rank == 0:
             print(json.dumps(run_reference(args, cfg)), flush=True)
         return
+    args.total_params = 0
+    if args.sharded and world > 1:
+        from dataclasses import replace
+        from paper_1511_05950_b200.sharded import shard_bounds
+        from workloads import layouts
+        args.total_params = cfg.layout().num_params
+        bounds = shard_bounds(args.total_params, world)
+        local_n = bounds[rank + 1] - bounds[rank]
+        cfg = replace(cfg, name="%s@shard%dof%d" % (cfg.name, rank, world), layout=lambda: layouts.flat(local_n))
     if args.sweep:
         if rank == 0:
             print(json.dumps(run_sweep(args)), flush=True)

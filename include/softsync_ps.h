@@ -137,6 +137,9 @@ int ps_bind_weight_mirror(ps_t *ps, void *mirror_bf16_dev);
  * num_params * gradient size; base 16-byte aligned) that ps_push_gradient_host copies into. */
 int ps_bind_staging(ps_t *ps, void *slots_dev, int64_t slot_bytes, int num_slots);
 
+/* Sets / reads one ps_option (the paper fixes none of them; they configure this implementation).
+ * Unknown keys, values out of range and changes that are only allowed while no gradient is pending
+ * return PS_ERR_INVALID_ARG and change nothing. */
 int ps_set_option(ps_t *ps, int key, int64_t value);
 int ps_get_option(ps_t *ps, int key, int64_t *value);
 

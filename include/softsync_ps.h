@@ -58,7 +58,7 @@ enum ps_option {
     PS_OPT_FUSE_T = 2,                    /* max groups applied by one kernel pass, 1..PS_MAX_FUSE_T (default 1) */
     PS_OPT_STREAM = 3,                    /* cudaStream_t as an integer (default 0) */
     PS_OPT_QUEUE_GROUPS = 4,              /* max complete-but-unapplied groups (default 64) */
-    PS_OPT_LOG_UPDATES = 5,               /* how many most recent updates the log keeps (default 65536) */
+    PS_OPT_LOG_UPDATES = 5,               /* how many most recent updates the log keeps (default max(1024, 2^20 / c)) */
     PS_OPT_TIMING = 6,                    /* 1: bracket every update kernel with CUDA events (ps_kernel_time) */
     PS_OPT_KERNEL = 7,                    /* ps_kernel_choice (default PS_KERNEL_AUTO) */
     PS_OPT_PROTOCOL = 10,                 /* ps_protocol (default PS_PROTOCOL_SOFTSYNC); only while nothing is pending */

@@ -50,7 +50,7 @@ struct ps_ctx {
     int fuse_t = 1;
     cudaStream_t stream = nullptr;
     int64_t queue_groups = 64;
-    int64_t log_updates = 65536;
+    int64_t log_updates = 65536;           // set in ps_create: about one million log entries
     int timing = 0, kernel_choice = PS_KERNEL_AUTO, block_threads = 0, overlap_launch = 0;
     int protocol = PS_PROTOCOL_SOFTSYNC;
     int sm_count = 0;
@@ -368,6 +368,7 @@ int ps_create(ps_t **out, int64_t num_params, int lambda, int n,
         ps->n = num_params; ps->lambda = lambda; ps->split = n; ps->c = lambda / n;   // Eq. 2: c = floor(lambda / n)
         ps->alpha0 = alpha0; ps->momentum = momentum; ps->weight_decay = weight_decay;
         ps->modulation = modulation;
+        ps->log_updates = std::max<int64_t>(1024, (int64_t{1} << 20) / ps->c);
         cudaError_t e = cudaGetDevice(&ps->device);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ps->sm_count, cudaDevAttrMultiProcessorCount, ps->device);
         if (e != cudaSuccess) {

@@ -183,6 +183,16 @@ int ps_push_gradient(ps_t *ps, int learner, const void *grad_dev, int64_t ts);
  * unchanged until the stream has passed the copy. */
 int ps_push_gradient_host(ps_t *ps, int learner, const void *grad_host, int64_t ts);
 
+/* Receive buffers for learners on the same GPU (the counterpart of the server-side receive buffer of the
+ * paper's MPI transport, Section 2.3): ps_acquire_slot lends one free staging slot (bound with
+ * ps_bind_staging); the learner writes its gradient there with its own kernels or copies, ordered before
+ * the update on the server's stream, and hands it over with ps_push_slot, which behaves like
+ * ps_push_gradient and returns the slot to the pool once the update that consumes it is enqueued.  A slot
+ * that will not be pushed goes back with ps_release_slot.  PS_ERR_QUEUE_FULL when every slot is in use. */
+int ps_acquire_slot(ps_t *ps, void **slot_dev, int *slot_id);
+int ps_push_slot(ps_t *ps, int learner, int slot_id, int64_t ts);
+int ps_release_slot(ps_t *ps, int slot_id);
+
 /* applyUpdate fused with sumGradients (Section 2.1; Eq. 2 with the learning rate of Eq. 3):
  * takes up to PS_OPT_FUSE_T complete groups, oldest first, and applies them in ONE kernel pass
  * that reads theta and v once, reads every gradient of those groups once, and writes theta and

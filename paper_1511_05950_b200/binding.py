@@ -42,7 +42,7 @@ EXPORTS = (
     "ps_create", "ps_destroy", "ps_bind_state", "ps_init_weights", "ps_bind_staging", "ps_bind_weight_mirror",
     "ps_pull_weights_bf16",
     "ps_set_option", "ps_get_option", "ps_set_alpha0", "ps_pull_weights", "ps_pull_weights_host", "ps_pull_weights_host_async",
-    "ps_push_gradient", "ps_push_gradient_host", "ps_apply_update", "ps_flush", "ps_synchronize",
+    "ps_push_gradient", "ps_push_gradient_host", "ps_acquire_slot", "ps_push_slot", "ps_release_slot", "ps_apply_update", "ps_flush", "ps_synchronize",
     "ps_get_update_log", "ps_peek_state", "ps_export_state", "ps_import_state", "ps_kernel_time", "ps_last_cuda_error", "ps_status_string",
 )
 
@@ -77,6 +77,9 @@ def _load() -> C.CDLL:
         "ps_pull_weights_host_async": [vp, vp, C.POINTER(i64)],
         "ps_push_gradient": [vp, i32, vp, i64],
         "ps_push_gradient_host": [vp, i32, vp, i64],
+        "ps_acquire_slot": [vp, C.POINTER(vp), C.POINTER(i32)],
+        "ps_push_slot": [vp, i32, i32, i64],
+        "ps_release_slot": [vp, i32],
         "ps_apply_update": [vp],
         "ps_flush": [vp],
         "ps_synchronize": [vp],
@@ -114,6 +117,9 @@ ps_pull_weights_host = lib.ps_pull_weights_host
 ps_pull_weights_host_async = lib.ps_pull_weights_host_async
 ps_push_gradient = lib.ps_push_gradient
 ps_push_gradient_host = lib.ps_push_gradient_host
+ps_acquire_slot = lib.ps_acquire_slot
+ps_push_slot = lib.ps_push_slot
+ps_release_slot = lib.ps_release_slot
 ps_apply_update = lib.ps_apply_update
 ps_flush = lib.ps_flush
 ps_synchronize = lib.ps_synchronize
@@ -275,6 +281,24 @@ class ParameterServer:
             if len(self._host_held) > 1024:
                 self.synchronize()
         return r == PS_READY
+
+    def acquire_slot(self, dtype: Optional[torch.dtype] = None):
+        """(slot id, tensor view of a server-owned receive slot) for a learner to write its gradient into."""
+        ptr, sid = C.c_void_p(), C.c_int()
+        _check(ps_acquire_slot(self._h, C.byref(ptr), C.byref(sid)), "ps_acquire_slot")
+        elem = 2 if self.grad_dtype == "bf16" else 4
+        off = ptr.value - self._staging.data_ptr()
+        view = self._staging[off: off + self.num_params * elem].view(
+            torch.bfloat16 if self.grad_dtype == "bf16" else torch.float32)
+        return sid.value, view
+
+    def push_slot(self, learner: int, slot_id: int, ts: int) -> bool:
+        r = _check(ps_push_slot(self._h, learner, slot_id, ts), "ps_push_slot")
+        self._held.append(None)
+        return r == PS_READY
+
+    def release_slot(self, slot_id: int) -> None:
+        _check(ps_release_slot(self._h, slot_id), "ps_release_slot")
 
     def apply_update(self) -> int:
         done = _check(ps_apply_update(self._h), "ps_apply_update")

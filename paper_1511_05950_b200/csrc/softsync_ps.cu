@@ -44,6 +44,7 @@ struct ps_ctx {
     char *staging = nullptr;
     int64_t slot_bytes = 0;
     std::vector<int> free_slots;
+    std::vector<char> slot_lent;           // 1 while a learner holds the slot between acquire and push
     int num_slots = 0;
 
     int grad_dtype = PS_GRAD_FP32;
@@ -473,6 +474,7 @@ int ps_bind_staging(ps_t *ps, void *slots_dev, int64_t slot_bytes, int num_slots
         ps->slot_bytes = slot_bytes; ps->num_slots = num_slots;
         ps->free_slots.clear();
         for (int s = num_slots - 1; s >= 0; --s) ps->free_slots.push_back(s);
+        ps->slot_lent.assign(num_slots, 0);
         return PS_OK;
     } PS_CATCH_ALL
 }
@@ -675,6 +677,43 @@ int ps_push_gradient_host(ps_t *ps, int learner, const void *grad_host, int64_t 
         if (bytes) PS_CUDA(ps, cudaMemcpyAsync(dst, grad_host, bytes, cudaMemcpyHostToDevice, ps->stream));
         ps->free_slots.pop_back();
         return push_common(ps, learner, dst, ts, slot);
+    } PS_CATCH_ALL
+}
+
+int ps_acquire_slot(ps_t *ps, void **slot_dev, int *slot_id)
+{
+    try {
+        if (!is_live(ps) || !slot_dev || !slot_id) return PS_ERR_INVALID_ARG;
+        if (!ps->staging) return PS_ERR_NO_STATE;
+        if (ps->free_slots.empty()) return PS_ERR_QUEUE_FULL;
+        const int slot = ps->free_slots.back();
+        ps->free_slots.pop_back();
+        ps->slot_lent[slot] = 1;
+        *slot_id = slot;
+        *slot_dev = ps->staging + static_cast<int64_t>(slot) * ps->slot_bytes;
+        return PS_OK;
+    } PS_CATCH_ALL
+}
+
+int ps_release_slot(ps_t *ps, int slot_id)
+{
+    try {
+        if (!is_live(ps) || slot_id < 0 || slot_id >= ps->num_slots || !ps->slot_lent[slot_id]) return PS_ERR_INVALID_ARG;
+        ps->slot_lent[slot_id] = 0;
+        ps->free_slots.push_back(slot_id);
+        return PS_OK;
+    } PS_CATCH_ALL
+}
+
+int ps_push_slot(ps_t *ps, int learner, int slot_id, int64_t ts)
+{
+    try {
+        if (!is_live(ps) || slot_id < 0 || slot_id >= ps->num_slots || !ps->slot_lent[slot_id]) return PS_ERR_INVALID_ARG;
+        const void *grad = ps->staging + static_cast<int64_t>(slot_id) * ps->slot_bytes;
+        const int rc = check_push(ps, learner, grad, ts);
+        if (rc != PS_OK) return rc;                       // the learner keeps the slot and may try again
+        ps->slot_lent[slot_id] = 0;
+        return push_common(ps, learner, grad, ts, slot_id);
     } PS_CATCH_ALL
 }
 

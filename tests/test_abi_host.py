@@ -285,6 +285,23 @@ def test_hardsync_mode_enforces_the_barrier():
     P.ps_destroy(h)
 
 
+def test_receive_slot_bookkeeping():
+    rc, h = make(2, 1)
+    ptr, sid, sid2 = C.c_void_p(), C.c_int(), C.c_int()
+    assert P.ps_acquire_slot(h, C.byref(ptr), C.byref(sid)) == P.PS_ERR_NO_STATE            # nothing bound
+    assert P.ps_bind_staging(h, 0x10000, 256, 2) == 0
+    assert P.ps_acquire_slot(h, C.byref(ptr), C.byref(sid)) == 0 and ptr.value in (0x10000, 0x10100)
+    assert P.ps_acquire_slot(h, C.byref(ptr), C.byref(sid2)) == 0 and sid2.value != sid.value
+    assert P.ps_acquire_slot(h, C.byref(ptr), C.byref(sid2)) == P.PS_ERR_QUEUE_FULL
+    assert P.ps_push_slot(h, 5, sid.value, 0) == P.PS_ERR_BAD_LEARNER                      # slot stays lent
+    assert P.ps_push_slot(h, 0, sid.value, 0) == P.PS_OK
+    assert P.ps_push_slot(h, 0, sid.value, 0) == P.PS_ERR_INVALID_ARG                      # already handed over
+    assert P.ps_release_slot(h, sid.value) == P.PS_ERR_INVALID_ARG
+    assert P.ps_release_slot(h, sid2.value) == 0
+    assert P.ps_release_slot(h, sid2.value) == P.PS_ERR_INVALID_ARG                        # not lent any more
+    P.ps_destroy(h)
+
+
 def test_status_strings():
     assert P.status_string(P.PS_ERR_BAD_TIMESTAMP).startswith("gradient timestamp")
     assert P.status_string(0) == "ok"

@@ -557,6 +557,36 @@ def test_asynchronous_host_pull_orders_with_later_updates():
     ps.destroy()
 
 
+def test_learners_write_into_server_owned_slots():
+    """Gradients produced straight into receive slots (acquire, write, push) give the same bits as borrowed buffers."""
+    dev = torch.device("cuda", 0)
+    n_el, lam = 20011, 3
+    w0 = G.initial_weights(layouts.flat(n_el), 41)
+    out = []
+    for use_slots in (False, True):
+        ps = P.ParameterServer(n_el, lam, 1, 0.02, 0.9, 5e-4, device=dev)
+        ps.init_weights(w0.to(dev))
+        if use_slots:
+            ps.bind_staging(lam + 1)
+        for u in range(5):
+            ts = ps.pull_weights()
+            for l in range(lam):
+                if use_slots:
+                    sid, view = ps.acquire_slot()
+                    G.gradient(41, l, u, n_el, 1e-3, device=dev, out=view)
+                    if l == 0 and u == 0:                                   # a slot can be handed back unused
+                        spare, _ = ps.acquire_slot()
+                        ps.release_slot(spare)
+                    fired = ps.push_slot(l, sid, ts)
+                else:
+                    fired = ps.push_gradient(l, G.gradient(41, l, u, n_el, 1e-3, device=dev), ts)
+            assert fired and ps.apply_update() == 1
+        ps.synchronize()
+        out.append((ps.w.cpu().numpy().copy(), ps.v.cpu().numpy().copy()))
+        ps.destroy()
+    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
+
+
 def test_staging_slots_run_out():
     dev = torch.device("cuda", 0)
     ps = P.ParameterServer(64, 4, 1, 0.01, device=dev)

@@ -28,6 +28,7 @@ MUTANTS = {
     "decay_unmodulated": ("update_rule.inc", "const REAL d = ROUND_SCALE(wd * S);", "const REAL d = ROUND_SCALE(wd * alpha0[0]);"),
     "rate_at_apply_time": ("softsync_oracle.c", "alpha0[l] = ps->pending[order[l]].alpha0;", "alpha0[l] = ps->alpha0;"),
     "barrier_lets_stale_in": ("softsync_oracle.c", "if (tau != 0) return -3;", "if (tau > 1) return -3;"),
+    "regrouped_sum": ("update_rule.inc", "const REAL t = acc + d * w[k];\n        v[k] = m * v[k] + t;", "v[k] = (m * v[k] + acc) + d * w[k];"),
     "staleness_plus_one": ("softsync_oracle.c", "sigma = tau > 0 ? tau : 1;", "sigma = tau + 1;"),
     "staleness_ignored": ("softsync_oracle.c", "sigma = tau > 0 ? tau : 1;", "sigma = 1;"),
     "clock_jumps": ("softsync_oracle.c", "ps->ts += 1;", "ps->ts += ps->c;"),
@@ -46,6 +47,7 @@ def _pins():
         TU.test_single_learner_matches_library_sgd_optimizer,
         lambda: TU.test_one_softsync_with_barrier_is_synchronous_averaged_sgd(4),
         TU.test_downpour_case_is_per_push_sgd,
+        TU.test_fp32_rounding_order_is_the_documented_one,
         TU.test_hardsync_protocol_is_eq_1_and_enforces_the_barrier,
         TU.test_step_schedule_without_momentum_is_library_sgd_with_a_changing_rate,
         TU.test_rate_in_force_at_arrival_enters_the_geometric_sum,

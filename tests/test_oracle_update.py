@@ -332,6 +332,42 @@ def test_decay_and_momentum_follow_the_linear_recurrence_in_matrix_form():
     assert tau.max() >= 3
 
 
+def test_fp32_rounding_order_is_the_documented_one():
+    """The fp32 state is rounded after every multiply and every add, in this order: products s_l*g_l summed
+    left to right in (learner, push) order; t = acc + d*w; v = m*v + t; w = w - v.  Written out with numpy
+    float32 scalars-as-arrays (each numpy op rounds once) and compared bit for bit on random data."""
+    lam, n, n_el, pushes = 6, 2, 301, 60
+    c = lam // n
+    f = np.float32
+    a0, m, wd = f(0.03), f(0.9), f(5e-4)
+    k, l = R.simulate_arrivals("lognormal", lam, pushes, 44)
+    tau, _ = staleness_by_recount(k, l, c)
+    w0 = G.normal_like(G.stream_key(44, G.STREAM_WEIGHTS), 0, n_el, 0.01).numpy()
+    ps = R.ReferencePS(n_el, lam, n, float(a0), float(m), float(wd), R.MOD_INV_STALENESS, 32)
+    ps.set_weights(w0)
+    arrivals_ = []
+    def grad(a, b):
+        g = G.gradient(44, a, b, n_el, 1e-3).numpy()
+        arrivals_.append((a, b, g))
+        return g
+    replay_reference(ps, k, l, grad)
+    w, v = w0.copy(), np.zeros(n_el, f)
+    for i in range(pushes // c):
+        group = sorted(((a, b, g, max(int(tau[i * c + j]), 1)) for j, (a, b, g) in enumerate(arrivals_[i * c:(i + 1) * c])),
+                       key=lambda x: (x[0], x[1]))
+        s = [f(np.float64(a0) / (np.float64(c) * np.float64(sig))) for _, _, _, sig in group]
+        d = f(np.float64(wd) * sum(np.float64(x) for x in s))
+        acc = s[0] * group[0][2]
+        for j in range(1, c):
+            acc = acc + s[j] * group[j][2]
+        t = acc + d * w
+        v = m * v + t
+        w = w - v
+    wr, vr = ps.state()
+    assert np.array_equal(wr.astype(f), w) and np.array_equal(vr.astype(f), v)
+    assert tau.max() >= 2
+
+
 # ---------------------------------------------------------------- invariants of the readings
 def test_arrival_order_inside_a_group_does_not_change_the_bits():
     lam, n_el = 5, 33

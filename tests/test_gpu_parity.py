@@ -446,6 +446,12 @@ def test_two_servers_on_their_own_streams():
         servers[k].destroy()
 
 
+@pytest.mark.parametrize("grad_dtype", ["fp32", "bf16"])
+def test_largest_launch_512_entries(grad_dtype):
+    """c = 256 (the largest group) with two groups fused: 512 gradient pointers in one launch."""
+    _simple(2051, 256, 1, 4 * 256, grad_dtype, model="uniform", fuse_t=16, lazy=True)
+
+
 def test_zero_parameters():
     _simple(0, 4, 2, 12)
 

@@ -118,7 +118,8 @@ int ps_destroy(ps_t *ps);
 
 /* Binds caller-owned device buffers of num_params fp32 each: weights theta and momentum v.
  * They must stay valid until ps_destroy.  4-byte alignment is enough; 16-byte alignment
- * enables the vector kernel.  Does not touch their contents. */
+ * enables the vector kernel.  Does not touch their contents (a bf16 mirror bound earlier is refilled
+ * from the new weights). */
 int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev);
 
 /* Sets theta_0 (copied from w_src, host memory if src_is_host != 0, else device), zeroes the

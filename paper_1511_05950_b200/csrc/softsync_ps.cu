@@ -419,8 +419,11 @@ int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev)
         if (!is_live(ps) || !w_dev || !v_dev || w_dev == v_dev) return PS_ERR_INVALID_ARG;
         if ((reinterpret_cast<uintptr_t>(w_dev) & 3u) || (reinterpret_cast<uintptr_t>(v_dev) & 3u)) return PS_ERR_INVALID_ARG;
         if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+        if (w_dev == reinterpret_cast<float *>(ps->mirror) || v_dev == reinterpret_cast<float *>(ps->mirror))
+            return PS_ERR_INVALID_ARG;
         ps->w = w_dev; ps->v = v_dev;
-        return PS_OK;
+        DeviceGuard on_device(ps);
+        return refresh_mirror(ps);                        // a mirror bound earlier follows the new theta
     } PS_CATCH_ALL
 }
 

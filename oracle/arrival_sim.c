@@ -19,7 +19,9 @@
  * Pins (tests/test_oracle_arrivals.py): with lambda = 30 homogeneous learners
  * the paper measures tau in {0,1,2} for 1-softsync and a mean staleness close
  * to n with nothing beyond 2n for n = 15, 30 (Section 2.4, Fig. 1); with
- * Exp(1) times and c = 1 the staleness is geometric with mean lambda - 1.
+ * Exp(1) times and c = 1 the staleness is geometric with mean lambda - 1; the
+ * log-normal model's per-learner mean duration has log-standard-deviation 0.5 and
+ * its durations spread +-5 % around that mean (checked on the simulated times).
  */
 #include <math.h>
 #include <stdint.h>
@@ -62,14 +64,14 @@ static double draw_duration(int model, double speed, uint64_t *state)
  * or -1 if cap is too small / arguments are invalid.  The trace opens with a
  * pull by every learner and ends with the pull that follows push number
  * num_pushes. */
-int64_t oracle_simulate_arrivals(int model, int lambda, int64_t num_pushes, uint64_t seed,
-                                 int32_t *kind, int32_t *learner, int64_t cap)
+static int64_t simulate(int model, int lambda, int64_t num_pushes, uint64_t seed,
+                        int32_t *kind, int32_t *learner, double *when, int64_t cap)
 {
     if (lambda < 1 || num_pushes < 0 || model < 0 || model > 3) return -1;
     if (cap < lambda + 2 * num_pushes) return -1;
     uint64_t state = seed;
     int64_t ne = 0, pushes = 0;
-    for (int l = 0; l < lambda; ++l) { kind[ne] = EV_PULL; learner[ne] = l; ++ne; }
+    for (int l = 0; l < lambda; ++l) { kind[ne] = EV_PULL; learner[ne] = l; if (when) when[ne] = 0.0; ++ne; }
 
     if (model == 0) {
         int *perm = malloc(sizeof(int) * lambda);
@@ -80,8 +82,8 @@ int64_t oracle_simulate_arrivals(int model, int lambda, int64_t num_pushes, uint
                 int t = perm[a]; perm[a] = perm[b]; perm[b] = t;
             }
             for (int a = 0; a < lambda && pushes < num_pushes; ++a, ++pushes) {
-                kind[ne] = EV_PUSH; learner[ne] = perm[a]; ++ne;
-                kind[ne] = EV_PULL; learner[ne] = perm[a]; ++ne;
+                kind[ne] = EV_PUSH; learner[ne] = perm[a]; if (when) when[ne] = (double)pushes; ++ne;
+                kind[ne] = EV_PULL; learner[ne] = perm[a]; if (when) when[ne] = (double)pushes; ++ne;
             }
         }
         free(perm);
@@ -95,10 +97,23 @@ int64_t oracle_simulate_arrivals(int model, int lambda, int64_t num_pushes, uint
     for (; pushes < num_pushes; ++pushes) {
         int first = 0;                                    /* earliest finisher, lowest id on ties */
         for (int l = 1; l < lambda; ++l) if (done[l] < done[first]) first = l;
-        kind[ne] = EV_PUSH; learner[ne] = first; ++ne;
-        kind[ne] = EV_PULL; learner[ne] = first; ++ne;
+        kind[ne] = EV_PUSH; learner[ne] = first; if (when) when[ne] = done[first]; ++ne;
+        kind[ne] = EV_PULL; learner[ne] = first; if (when) when[ne] = done[first]; ++ne;
         done[first] += draw_duration(model, speed[first], &state);
     }
     free(done); free(speed);
     return ne;
+}
+
+int64_t oracle_simulate_arrivals(int model, int lambda, int64_t num_pushes, uint64_t seed,
+                                 int32_t *kind, int32_t *learner, int64_t cap)
+{
+    return simulate(model, lambda, num_pushes, seed, kind, learner, NULL, cap);
+}
+
+/* The same trace together with the simulated time of every event (for checking the duration laws). */
+int64_t oracle_simulate_arrivals_timed(int model, int lambda, int64_t num_pushes, uint64_t seed,
+                                       int32_t *kind, int32_t *learner, double *when, int64_t cap)
+{
+    return simulate(model, lambda, num_pushes, seed, kind, learner, when, cap);
 }

@@ -15,6 +15,7 @@ from . import build as _build
 
 MOD_CONSTANT = 0
 MOD_INV_STALENESS = 1
+MOD_EXP_STALENESS = 2
 GRAD_FP32 = 0
 GRAD_BF16 = 1
 
@@ -40,6 +41,8 @@ def load(path: str) -> C.CDLL:
         L.oracle_ps_set_weights.argtypes = [C.c_void_p, C.c_void_p]
         L.oracle_ps_set_alpha0.argtypes = [C.c_void_p, C.c_float]
         L.oracle_ps_set_hardsync.argtypes = [C.c_void_p, C.c_int]
+        L.oracle_ps_set_penalty_base.argtypes = [C.c_void_p, C.c_float]
+        L.oracle_ps_set_layer_multipliers.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         L.oracle_ps_timestamp.restype = C.c_int64
         L.oracle_ps_timestamp.argtypes = [C.c_void_p]
         L.oracle_ps_group_size.argtypes = [C.c_void_p]
@@ -55,6 +58,9 @@ def load(path: str) -> C.CDLL:
         L.oracle_ps_get_log.argtypes = [C.c_void_p, C.c_void_p]
         L.oracle_simulate_arrivals.restype = C.c_int64
         L.oracle_simulate_arrivals.argtypes = [C.c_int, C.c_int, C.c_int64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_int64]
+        L.oracle_simulate_arrivals_timed.restype = C.c_int64
+        L.oracle_simulate_arrivals_timed.argtypes = [C.c_int, C.c_int, C.c_int64, C.c_uint64, C.c_void_p, C.c_void_p,
+                                                     C.c_void_p, C.c_int64]
         assert LOG_DTYPE.itemsize == 64
     return L
 
@@ -88,6 +94,19 @@ def simulate_arrivals(model: str, num_learners: int, num_pushes: int, seed: int)
     if n < 0:
         raise ValueError("oracle_simulate_arrivals rejected its arguments")
     return kind[:n].copy(), learner[:n].copy()
+
+
+def simulate_arrivals_timed(model: str, num_learners: int, num_pushes: int, seed: int):
+    """(kind, learner, simulated time) of the same trace simulate_arrivals returns."""
+    cap = num_learners + 2 * num_pushes
+    kind = np.empty(cap, dtype=np.int32)
+    learner = np.empty(cap, dtype=np.int32)
+    when = np.empty(cap, dtype=np.float64)
+    n = lib().oracle_simulate_arrivals_timed(ARRIVAL_MODELS[model], num_learners, num_pushes, seed,
+                                             kind.ctypes.data, learner.ctypes.data, when.ctypes.data, cap)
+    if n < 0:
+        raise ValueError("oracle_simulate_arrivals_timed rejected its arguments")
+    return kind[:n].copy(), learner[:n].copy(), when[:n].copy()
 
 
 def round_to_bf16(x: np.ndarray) -> np.ndarray:
@@ -127,6 +146,22 @@ class ReferencePS:
         """Switch to the hardsync protocol (needs n = 1, nothing pending)."""
         if lib().oracle_ps_set_hardsync(self._h, int(on)) != 0:
             raise ValueError("hardsync needs n = 1 and no pending gradient")
+
+    def set_penalty_base(self, rho: float) -> None:
+        """Base of the exponential staleness penalty alpha0 * rho**tau (MOD_EXP_STALENESS)."""
+        if lib().oracle_ps_set_penalty_base(self._h, rho) != 0:
+            raise ValueError("penalty base must lie in (0, 1]")
+
+    def set_layer_multipliers(self, bounds, lr_mult, wd_mult) -> None:
+        """Layer q = elements [bounds[q], bounds[q+1]) with learning-rate and decay multipliers."""
+        bounds = np.ascontiguousarray(bounds, dtype=np.int64)
+        lr_mult = np.ascontiguousarray(lr_mult, dtype=np.float32)
+        wd_mult = np.ascontiguousarray(wd_mult, dtype=np.float32)
+        nseg = lr_mult.size
+        assert wd_mult.size == nseg and bounds.size == nseg + 1
+        if lib().oracle_ps_set_layer_multipliers(self._h, nseg, bounds.ctypes.data, lr_mult.ctypes.data,
+                                                 wd_mult.ctypes.data) != 0:
+            raise ValueError("layer bounds must tile [0, num_params)")
 
     def set_alpha0(self, alpha0: float) -> None:
         """Base learning rate for gradients pushed from now on."""

@@ -26,15 +26,20 @@
  *   - the update runs inside the push that completes the group; a pull that
  *     follows sees the new clock.
  *   - momentum and weight decay: see update_rule.inc.
+ *   - exponential penalty (the earlier proposal that Section 1 sets the 1/tau rule against; the
+ *     paper gives no formula for it): alpha = alpha0 * rho^tau with a base 0 < rho <= 1, so a fresh
+ *     gradient (tau = 0) gets alpha0; the log's sigma field then holds tau itself.
+ *   - per-layer multipliers: see update_rule.inc.
  *   - the base rate alpha0 may be changed between calls (the step schedules of
  *     Section 4.3); a gradient is scaled with the alpha0 in force when it arrived,
- *     since Section 2.4 sets the rate "for an incoming gradient".
+ *     since Section 2.4 (Eq. 3) fixes the rate per gradient as it comes in.
  *
  * Parity pins: tests/test_oracle_*.py (hand-worked examples under
  * tests/golden/, closed forms, reductions to plain SGD, invariants).
  * Convergence/accuracy behaviour of the method is not modelled here:
  * parity unpinned for it (it needs the paper's datasets).
  */
+#include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
@@ -43,6 +48,7 @@
 
 #define ORACLE_MOD_CONSTANT 0
 #define ORACLE_MOD_INV_STALENESS 1
+#define ORACLE_MOD_EXP_STALENESS 2
 
 #define ORACLE_GRAD_FP32 0
 #define ORACLE_GRAD_BF16 1
@@ -89,6 +95,8 @@ typedef struct oracle_ps {
     int lambda, n, c, modulation, precision;
     int hardsync;                    /* 1: the hardsync protocol of Section 2.2 (barrier, staleness 0) */
     double alpha0, momentum, wd;     /* exact widenings of the fp32 parameters */
+    double rho;                      /* base of the exponential staleness penalty */
+    float *lm, *dm;                  /* per-element rate / decay multipliers, NULL = all 1 */
     void *w, *v;
     int64_t ts;
     int64_t *pulled_ts;              /* -1: has not pulled yet */
@@ -106,12 +114,14 @@ oracle_ps *oracle_ps_create(int64_t N, int lambda, int n, float alpha0, float mo
 {
     if (N < 0 || lambda < 1 || n < 1 || n > lambda) return NULL;
     if (precision != 32 && precision != 64) return NULL;
+    if (modulation < ORACLE_MOD_CONSTANT || modulation > ORACLE_MOD_EXP_STALENESS) return NULL;
     if (lambda / n > ORACLE_MAX_C) return NULL;
     oracle_ps *ps = calloc(1, sizeof *ps);
     ps->N = N; ps->lambda = lambda; ps->n = n;
     ps->c = lambda / n;                                   /* Eq. 2: c = floor(lambda/n) */
     ps->alpha0 = alpha0; ps->momentum = momentum; ps->wd = weight_decay;
     ps->modulation = modulation; ps->precision = precision;
+    ps->rho = 0.5;
     ps->w = calloc((size_t)(N ? N : 1), real_size(ps));
     ps->v = calloc((size_t)(N ? N : 1), real_size(ps));
     ps->pulled_ts = malloc(sizeof(int64_t) * lambda);
@@ -127,7 +137,7 @@ void oracle_ps_destroy(oracle_ps *ps)
     if (!ps) return;
     for (int l = 0; l < ps->c; ++l) free(ps->pending[l].grad);
     free(ps->pending); free(ps->w); free(ps->v);
-    free(ps->pulled_ts); free(ps->push_count); free(ps->log); free(ps);
+    free(ps->pulled_ts); free(ps->push_count); free(ps->log); free(ps->lm); free(ps->dm); free(ps);
 }
 
 /* theta_0 = w0, velocity 0, clock 0 (Section 2.1). */
@@ -148,6 +158,33 @@ int oracle_ps_set_hardsync(oracle_ps *ps, int on)
     if (on && ps->n != 1) return -1;
     if (ps->npending) return -1;
     ps->hardsync = on ? 1 : 0;
+    return 0;
+}
+
+/* Base rho of the exponential staleness penalty alpha0 * rho^tau (0 < rho <= 1); used only when the
+ * server was created with ORACLE_MOD_EXP_STALENESS.  Returns 0, or -1 for a base outside (0, 1]. */
+int oracle_ps_set_penalty_base(oracle_ps *ps, float rho)
+{
+    if (!(rho > 0.0f) || rho > 1.0f) return -1;
+    ps->rho = rho;
+    return 0;
+}
+
+/* Per-layer multipliers: layer q covers elements [bounds[q], bounds[q+1]) (bounds[0] = 0,
+ * bounds[nseg] = N, ascending) and scales the learning rate by lr_mult[q] and the weight decay by
+ * wd_mult[q].  nseg = 0 removes them.  Returns 0, or -1 if the bounds do not tile [0, N). */
+int oracle_ps_set_layer_multipliers(oracle_ps *ps, int nseg, const int64_t *bounds,
+                                    const float *lr_mult, const float *wd_mult)
+{
+    if (nseg < 0) return -1;
+    if (nseg == 0) { free(ps->lm); free(ps->dm); ps->lm = ps->dm = NULL; return 0; }
+    if (bounds[0] != 0 || bounds[nseg] != ps->N) return -1;
+    for (int q = 0; q < nseg; ++q) if (bounds[q] > bounds[q + 1]) return -1;
+    free(ps->lm); free(ps->dm);
+    ps->lm = malloc(sizeof(float) * (size_t)(ps->N ? ps->N : 1));
+    ps->dm = malloc(sizeof(float) * (size_t)(ps->N ? ps->N : 1));
+    for (int q = 0; q < nseg; ++q)
+        for (int64_t k = bounds[q]; k < bounds[q + 1]; ++k) { ps->lm[k] = lr_mult[q]; ps->dm[k] = wd_mult[q]; }
     return 0;
 }
 
@@ -198,20 +235,22 @@ static void apply_pending(oracle_ps *ps)
         order[b + 1] = x;
     }
     const void *grads[ORACLE_MAX_C];
-    int64_t sigma[ORACLE_MAX_C];
+    int64_t sigma[ORACLE_MAX_C], tau[ORACLE_MAX_C];
     double scale[ORACLE_MAX_C], alpha0[ORACLE_MAX_C];
     for (int l = 0; l < c; ++l) {
         grads[l] = ps->pending[order[l]].grad; sigma[l] = ps->pending[order[l]].sigma;
+        tau[l] = ps->pending[order[l]].tau;
         alpha0[l] = ps->pending[order[l]].alpha0;
     }
+    const int exp_penalty = ps->modulation == ORACLE_MOD_EXP_STALENESS;
 
     double d;
     if (ps->precision == 32)
-        d = apply_group_f32(ps->w, ps->v, ps->N, c, (const float *const *)grads, sigma,
-                            alpha0, ps->momentum, ps->wd, scale);
+        d = apply_group_f32(ps->w, ps->v, ps->N, c, (const float *const *)grads, sigma, tau,
+                            alpha0, exp_penalty, ps->rho, ps->momentum, ps->wd, ps->lm, ps->dm, scale);
     else
-        d = apply_group_f64(ps->w, ps->v, ps->N, c, (const double *const *)grads, sigma,
-                            alpha0, ps->momentum, ps->wd, scale);
+        d = apply_group_f64(ps->w, ps->v, ps->N, c, (const double *const *)grads, sigma, tau,
+                            alpha0, exp_penalty, ps->rho, ps->momentum, ps->wd, ps->lm, ps->dm, scale);
 
     for (int l = 0; l < c; ++l) {
         const pending_t *p = &ps->pending[order[l]];
@@ -241,6 +280,8 @@ int oracle_ps_push_with_timestamp(oracle_ps *ps, int learner, const void *grad, 
     int64_t sigma = 1;
     if (ps->modulation == ORACLE_MOD_INV_STALENESS)
         sigma = tau > 0 ? tau : 1;                       /* Eq. 3, and alpha0 itself at tau = 0 */
+    if (ps->modulation == ORACLE_MOD_EXP_STALENESS)
+        sigma = tau;                                     /* the penalty's exponent */
 
     pending_t *p = &ps->pending[ps->npending++];
     p->learner = learner; p->push_index = ps->push_count[learner]++;

@@ -64,6 +64,41 @@ def test_lognormal_speeds_are_heavy_tailed():
     assert pushes_per_learner.max() > 3 * max(1, pushes_per_learner.min())
 
 
+def test_lognormal_model_has_the_stated_speed_and_jitter_laws():
+    """Persistent speed exp(0.5 z), z ~ N(0,1), times a per-iteration jitter U[0.95, 1.05]: measured on the
+    simulated times.  The log of a learner's mean iteration time has standard deviation 0.5 (a shape
+    parameter of 1.0 or 0.25 fails), is symmetric and normal-shaped; every iteration lies within 5 % of the
+    learner's speed, uniformly (standard deviation 0.1/sqrt(12))."""
+    lam, pushes = 1500, 150000
+    k, l, t = R.simulate_arrivals_timed("lognormal", lam, pushes, 77)
+    k2, l2 = R.simulate_arrivals("lognormal", lam, pushes, 77)
+    assert np.array_equal(k, k2) and np.array_equal(l, l2)             # the timed form is the same trace
+    push = k == R.PUSH
+    assert (np.diff(t[push]) >= 0).all()                                # the server serves in time order
+    speeds, rel = [], []
+    for who in range(lam):
+        times = t[push & (l == who)]
+        if times.size < 12:
+            continue
+        dur = np.diff(np.concatenate([[0.0], times]))
+        centre = 0.5 * (dur.max() + dur.min())                          # jitter is symmetric about the speed
+        speeds.append(dur.mean())
+        rel.append(dur / centre)
+    z = np.log(np.asarray(speeds))
+    assert len(speeds) > 0.9 * lam
+    rel = np.concatenate(rel)
+    assert rel.min() > 0.94 and rel.max() < 1.06
+    assert abs(rel.std() - 0.1 / np.sqrt(12)) < 0.003
+    # slow learners drop out of the sample above (fewer than 12 pushes), which trims the upper tail a little
+    assert 0.42 < z.std() < 0.53
+    inside = (np.abs(z - np.median(z)) < 0.5).mean()
+    assert 0.62 < inside < 0.75                                          # 68 % within one shape parameter
+    # more pushes from faster learners, in proportion to 1 / speed
+    counts = np.bincount(l[push], minlength=lam)
+    fast, slow = counts[np.argsort(counts)[-50:]].mean(), counts[np.argsort(counts)[:50]].mean()
+    assert fast > 4 * slow
+
+
 @pytest.mark.parametrize("model,lam,n", [("exp", 7, 3), ("uniform", 18, 4), ("lognormal", 9, 9), ("rounds", 5, 1)])
 def test_clock_and_staleness_against_brute_force_recount(model, lam, n):
     pushes = 500

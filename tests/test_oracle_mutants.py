@@ -18,17 +18,24 @@ from tests import test_oracle_update as TU
 ORACLE_DIR = os.path.dirname(os.path.abspath(R.__file__))
 
 MUTANTS = {
-    "decay_sign": ("update_rule.inc", "const REAL t = acc + d * w[k];", "const REAL t = acc - d * w[k];"),
+    "decay_sign": ("update_rule.inc", "REAL t = acc + dk * w[k];", "REAL t = acc - dk * w[k];"),
     "descent_sign": ("update_rule.inc", "w[k] = w[k] - v[k];", "w[k] = w[k] + v[k];"),
     "momentum_dropped": ("update_rule.inc", "v[k] = m * v[k] + t;", "v[k] = t;"),
-    "decay_dropped": ("update_rule.inc", "const REAL t = acc + d * w[k];", "const REAL t = acc;"),
+    "decay_dropped": ("update_rule.inc", "REAL t = acc + dk * w[k];", "REAL t = acc;"),
     "no_averaging": ("update_rule.inc", "((double)c * (double)sigma[l])", "((double)sigma[l])"),
     "wrong_gradient_index": ("update_rule.inc", "acc = acc + s[l] * grads[l][k];", "acc = acc + s[l] * grads[0][k];"),
     "wrong_scale_index": ("update_rule.inc", "acc = acc + s[l] * grads[l][k];", "acc = acc + s[0] * grads[l][k];"),
     "decay_unmodulated": ("update_rule.inc", "const REAL d = ROUND_SCALE(wd * S);", "const REAL d = ROUND_SCALE(wd * alpha0[0]);"),
     "rate_at_apply_time": ("softsync_oracle.c", "alpha0[l] = ps->pending[order[l]].alpha0;", "alpha0[l] = ps->alpha0;"),
     "barrier_lets_stale_in": ("softsync_oracle.c", "if (tau != 0) return -3;", "if (tau > 1) return -3;"),
-    "regrouped_sum": ("update_rule.inc", "const REAL t = acc + d * w[k];\n        v[k] = m * v[k] + t;", "v[k] = (m * v[k] + acc) + d * w[k];"),
+    "regrouped_sum": ("update_rule.inc", "v[k] = m * v[k] + t;", "v[k] = (m * v[k] + acc) + (t - acc);"),
+    "penalty_linear_in_staleness": ("update_rule.inc", "pow(rho, (double)tau[l])", "(1.0 - (1.0 - rho) * (double)tau[l])"),
+    "penalty_not_averaged": ("update_rule.inc", "pow(rho, (double)tau[l]) / (double)c", "pow(rho, (double)tau[l])"),
+    "penalty_counts_one_more": ("update_rule.inc", "pow(rho, (double)tau[l])", "pow(rho, (double)tau[l] + 1.0)"),
+    "multipliers_swapped": ("update_rule.inc", "if (dm) dk = (REAL)dm[k] * d;", "if (dm) dk = (REAL)lm[k] * d;"),
+    "rate_multiplier_skips_decay": ("update_rule.inc", "if (lm) t = (REAL)lm[k] * t;", "if (lm) t = (REAL)lm[k] * acc + dk * w[k];"),
+    "decay_multiplier_dropped": ("update_rule.inc", "if (dm) dk = (REAL)dm[k] * d;", ""),
+    "layer_bound_off_by_one": ("softsync_oracle.c", "for (int64_t k = bounds[q]; k < bounds[q + 1]; ++k) {", "for (int64_t k = bounds[q] + (q > 0); k < bounds[q + 1] + (q + 1 < nseg); ++k) {"),
     "staleness_plus_one": ("softsync_oracle.c", "sigma = tau > 0 ? tau : 1;", "sigma = tau + 1;"),
     "staleness_ignored": ("softsync_oracle.c", "sigma = tau > 0 ? tau : 1;", "sigma = 1;"),
     "clock_jumps": ("softsync_oracle.c", "ps->ts += 1;", "ps->ts += ps->c;"),
@@ -52,6 +59,10 @@ def _pins():
         TU.test_step_schedule_without_momentum_is_library_sgd_with_a_changing_rate,
         TU.test_rate_in_force_at_arrival_enters_the_geometric_sum,
         lambda: TU.test_plain_rule_is_a_weighted_sum_of_gradients("exp", 12, 3),
+        lambda: TU.test_exponential_penalty_is_a_weighted_sum_with_geometric_weights(0.8),
+        TU.test_layer_multipliers_are_per_layer_rates_and_decays_of_library_sgd,
+        TU.test_layer_multipliers_of_one_change_nothing_and_zero_rate_freezes_a_layer,
+        TU.test_layer_multipliers_fp32_rounding_order,
         TU.test_momentum_is_a_geometric_sum_of_past_steps,
         TU.test_decay_and_momentum_follow_the_linear_recurrence_in_matrix_form,
         TU.test_arrival_order_inside_a_group_does_not_change_the_bits,

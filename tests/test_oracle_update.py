@@ -16,7 +16,7 @@ from tests.helpers import replay_reference, staleness_by_recount, rel_l2
 from workloads import generators as G
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "worked_softsync.json")
-MODS = {"inv_staleness": R.MOD_INV_STALENESS, "constant": R.MOD_CONSTANT}
+MODS = {"inv_staleness": R.MOD_INV_STALENESS, "constant": R.MOD_CONSTANT, "exp_staleness": R.MOD_EXP_STALENESS}
 
 
 def _grads(seed, lam, pushes_per_learner, n, std=1e-3, dtype=torch.float32):
@@ -31,6 +31,10 @@ def test_hand_worked_examples_exact(example, precision):
     ps = R.ReferencePS(len(ex["w0"]), ex["num_learners"], ex["n"], ex["alpha0"], ex["momentum"],
                        ex["weight_decay"], MODS[ex["modulation"]], precision)
     ps.set_weights(np.asarray(ex["w0"], np.float32))
+    if "penalty_base" in ex:
+        ps.set_penalty_base(ex["penalty_base"])
+    if "layers" in ex:
+        ps.set_layer_multipliers(ex["layers"]["bounds"], ex["layers"]["lr_mult"], ex["layers"]["wd_mult"])
     done = 0
     for ev in ex["events"]:
         if ev[0] == "pull":
@@ -270,6 +274,151 @@ def test_plain_rule_is_a_weighted_sum_of_gradients(model, lam, n):
     expect = w0.astype(np.float64) - np.einsum("p,pk->k", weights, np.stack(seen[:used]))
     assert rel_l2(ps.state()[0], expect) < 1e-13
     assert tau.max() >= 2       # the case really exercises staleness
+
+
+@pytest.mark.parametrize("rho", [0.5, 0.8, 1.0])
+def test_exponential_penalty_is_a_weighted_sum_with_geometric_weights(rho):
+    """m = 0, wd = 0 under the exponential penalty: theta_K = theta_0 - sum over pushes of
+    alpha0 * rho^tau / c * dtheta, with tau recounted from the raw trace; rho = 1 is the constant rate."""
+    lam, n, n_el, pushes = 12, 3, 40, 240
+    c = lam // n
+    a0, rho = float(np.float32(0.03)), float(np.float32(rho))
+    k, l = R.simulate_arrivals("exp", lam, pushes, 19)
+    tau, _ = staleness_by_recount(k, l, c)
+    ps = R.ReferencePS(n_el, lam, n, a0, 0.0, 0.0, R.MOD_EXP_STALENESS, 64)
+    ps.set_penalty_base(rho)
+    w0 = G.normal_like(G.stream_key(5, G.STREAM_WEIGHTS), 0, n_el, 0.01).numpy()
+    ps.set_weights(w0)
+    seen = []
+    def grad(a, b):
+        g = G.gradient(5, a, b, n_el, 1e-3).numpy()
+        seen.append(g.astype(np.float64))
+        return g
+    replay_reference(ps, k, l, grad)
+    used = (pushes // c) * c
+    weights = a0 * np.exp(np.log(rho) * tau[:used]) / c
+    expect = w0.astype(np.float64) - np.einsum("p,pk->k", weights, np.stack(seen[:used]))
+    assert rel_l2(ps.state()[0], expect) < 1e-12
+    assert tau.max() >= 3
+    log = ps.log()
+    assert np.array_equal(log["sigma"], log["tau"])
+    if rho == 1.0:                                     # no penalty at all: the constant-rate control of Section 4.3
+        const = R.ReferencePS(n_el, lam, n, a0, 0.0, 0.0, R.MOD_CONSTANT, 64)
+        const.set_weights(w0)
+        replay_reference(const, k, l, lambda a, b: G.gradient(5, a, b, n_el, 1e-3).numpy())
+        assert np.array_equal(const.state()[0], ps.state()[0])
+    with pytest.raises(ValueError):
+        ps.set_penalty_base(0.0)
+    with pytest.raises(ValueError):
+        ps.set_penalty_base(1.5)
+
+
+def test_exponential_penalty_shrinks_faster_than_inverse_staleness():
+    """Section 1's objection to the exponential rule: at the staleness a large system sees, it leaves almost
+    no step at all, whereas alpha0/tau decays only harmonically.  One gradient with tau = 40."""
+    out = {}
+    for mod in (R.MOD_INV_STALENESS, R.MOD_EXP_STALENESS):
+        ps = R.ReferencePS(1, 2, 2, 1.0, 0.0, 0.0, mod, 64)
+        ps.set_weights(np.zeros(1, np.float32))
+        ps.pull(0); ps.pull(1)
+        for _ in range(40):
+            ps.pull(0)
+            ps.push(0, np.zeros(1, np.float32))
+        ps.push(1, np.ones(1, np.float32))            # pulled at clock 0, arrives at clock 40
+        out[mod] = -ps.state()[0][0]
+        assert ps.log()["tau"][-1] == 40
+    assert out[R.MOD_INV_STALENESS] == 1.0 / 40
+    assert out[R.MOD_EXP_STALENESS] == 0.5 ** 40
+
+
+def _caffe_like_layers(n_el):
+    b = [0, n_el // 3, n_el // 3 + 5, n_el - 7, n_el]
+    return b, [1.0, 2.0, 0.5, 2.0], [1.0, 0.0, 3.0, 0.0]
+
+
+def test_layer_multipliers_are_per_layer_rates_and_decays_of_library_sgd():
+    """One learner: the method with multipliers (lm_q, dm_q) is library momentum SGD with one parameter
+    group per layer, lr = alpha0*lm_q and weight_decay = wd*dm_q (velocity here = lr * the library's buffer)."""
+    n_el, steps = 60, 50
+    f32 = lambda x: float(np.float32(x))
+    lr, m, wd = f32(0.01), f32(0.9), f32(5e-3)
+    bounds, lmul, dmul = _caffe_like_layers(n_el)
+    w0 = G.normal_like(G.stream_key(21, G.STREAM_WEIGHTS), 0, n_el, 0.1)
+    ps = R.ReferencePS(n_el, 1, 1, lr, m, wd, R.MOD_INV_STALENESS, 64)
+    ps.set_weights(w0.numpy())
+    ps.set_layer_multipliers(bounds, lmul, dmul)
+    params = [torch.nn.Parameter(w0[a:b].double().clone()) for a, b in zip(bounds[:-1], bounds[1:])]
+    opt = torch.optim.SGD([{"params": [p], "lr": lr * a, "weight_decay": wd * d} for p, a, d in zip(params, lmul, dmul)],
+                          lr=lr, momentum=m)
+    for s in range(steps):
+        g = G.gradient(21, 0, s, n_el, 1e-2)
+        ps.pull(0)
+        ps.push(0, g.numpy())
+        for p, a, b in zip(params, bounds[:-1], bounds[1:]):
+            p.grad = g[a:b].double()
+        opt.step()
+    w, v = ps.state()
+    assert rel_l2(w, torch.cat([p.detach() for p in params]).numpy()) < 1e-12
+    buf = torch.cat([opt.state[p]["momentum_buffer"] * (lr * a) for p, a in zip(params, lmul)]).numpy()
+    assert rel_l2(v, buf) < 1e-11
+
+
+def test_layer_multipliers_of_one_change_nothing_and_zero_rate_freezes_a_layer():
+    """Multiplying by 1.0f is exact, so all-ones multipliers give the same bits as none (fp32, real staleness);
+    a layer with rate multiplier 0 never moves."""
+    lam, n, n_el, pushes = 6, 2, 101, 60
+    k, l = R.simulate_arrivals("lognormal", lam, pushes, 4)
+    w0 = G.normal_like(G.stream_key(22, G.STREAM_WEIGHTS), 0, n_el, 0.01).numpy()
+    grad = lambda a, b: G.gradient(22, a, b, n_el, 1e-3).numpy()
+    out = []
+    for layers in (None, ([0, 40, n_el], [1.0, 1.0], [1.0, 1.0]), ([0, 40, n_el], [1.0, 0.0], [1.0, 1.0])):
+        ps = R.ReferencePS(n_el, lam, n, 0.03, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+        ps.set_weights(w0)
+        if layers:
+            ps.set_layer_multipliers(*layers)
+        replay_reference(ps, k, l, grad)
+        out.append(ps.state())
+    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
+    assert np.array_equal(out[2][0][:40], out[0][0][:40])
+    assert np.array_equal(out[2][0][40:].astype(np.float32), w0[40:]) and not out[2][1][40:].any()
+    with pytest.raises(ValueError):
+        R.ReferencePS(10, 1, 1, 0.1, 0.0, 0.0).set_layer_multipliers([0, 4, 9], [1, 1], [1, 1])   # does not reach N
+
+
+def test_layer_multipliers_fp32_rounding_order():
+    """t = lm * (acc + (dm * d) * w): every product and sum rounded once, written out in numpy float32."""
+    lam, n, n_el, pushes = 4, 2, 67, 24
+    c = lam // n
+    f = np.float32
+    a0, m, wd = f(0.03), f(0.9), f(5e-3)
+    bounds, lmul, dmul = _caffe_like_layers(n_el)
+    lm = np.repeat(np.asarray(lmul, f), np.diff(bounds)); dm = np.repeat(np.asarray(dmul, f), np.diff(bounds))
+    k, l = R.simulate_arrivals("exp", lam, pushes, 45)
+    tau, _ = staleness_by_recount(k, l, c)
+    w0 = G.normal_like(G.stream_key(45, G.STREAM_WEIGHTS), 0, n_el, 0.01).numpy()
+    ps = R.ReferencePS(n_el, lam, n, float(a0), float(m), float(wd), R.MOD_INV_STALENESS, 32)
+    ps.set_weights(w0)
+    ps.set_layer_multipliers(bounds, lmul, dmul)
+    arr = []
+    def grad(a, b):
+        g = G.gradient(45, a, b, n_el, 1e-3).numpy()
+        arr.append((a, b, g))
+        return g
+    replay_reference(ps, k, l, grad)
+    w, v = w0.copy(), np.zeros(n_el, f)
+    for i in range(pushes // c):
+        group = sorted(((a, b, g, max(int(tau[i * c + j]), 1)) for j, (a, b, g) in enumerate(arr[i * c:(i + 1) * c])),
+                       key=lambda x: (x[0], x[1]))
+        s = [f(np.float64(a0) / (np.float64(c) * np.float64(sig))) for _, _, _, sig in group]
+        d = f(np.float64(wd) * sum(np.float64(x) for x in s))
+        acc = s[0] * group[0][2]
+        for j in range(1, c):
+            acc = acc + s[j] * group[j][2]
+        t = lm * (acc + (dm * d) * w)
+        v = m * v + t
+        w = w - v
+    wr, vr = ps.state()
+    assert np.array_equal(wr.astype(f), w) and np.array_equal(vr.astype(f), v)
 
 
 def test_momentum_is_a_geometric_sum_of_past_steps():

@@ -33,7 +33,9 @@ typedef struct ps_ctx ps_t;               /* opaque; created by ps_create, freed
 
 enum ps_modulation {
     PS_MOD_CONSTANT = 0,                  /* alpha = alpha0 for every gradient (Section 4.3, case (a)) */
-    PS_MOD_INV_STALENESS = 1              /* alpha = alpha0 / max(tau, 1)       (Eq. 3; alpha0 at tau = 0) */
+    PS_MOD_INV_STALENESS = 1,             /* alpha = alpha0 / max(tau, 1)       (Eq. 3; alpha0 at tau = 0) */
+    PS_MOD_EXP_STALENESS = 2              /* alpha = alpha0 * rho^tau: the exponential penalty of the earlier work
+                                           * that Section 1 compares Eq. 3 with; rho: ps_set_penalty_base */
 };
 
 enum ps_status {
@@ -48,7 +50,9 @@ enum ps_status {
     PS_ERR_NOMEM = -7,                    /* host allocation failed */
     PS_ERR_NO_STATE = -8,                 /* weights/momentum (or staging slots) not bound yet */
     PS_ERR_LOG_EVICTED = -9,              /* requested log range is no longer (or not yet) held */
-    PS_ERR_BARRIER = -10                  /* hardsync: this learner has already contributed to the current round */
+    PS_ERR_BARRIER = -10,                 /* hardsync: this learner has already contributed to the current round */
+    PS_ERR_DEVICE_WAIT = -11              /* a bounded wait inside an update kernel ran out (PS_KERNEL_BULK); theta and v
+                                           * are partly updated and must be re-initialised; see ps_kernel_status */
 };
 
 enum ps_grad_dtype { PS_GRAD_FP32 = 0, PS_GRAD_BF16 = 1 };
@@ -56,14 +60,29 @@ enum ps_grad_dtype { PS_GRAD_FP32 = 0, PS_GRAD_BF16 = 1 };
 enum ps_option {
     PS_OPT_GRAD_DTYPE = 1,                /* ps_grad_dtype of every pushed gradient; only while nothing is pending */
     PS_OPT_FUSE_T = 2,                    /* max groups applied by one kernel pass, 1..PS_MAX_FUSE_T (default 1) */
-    PS_OPT_STREAM = 3,                    /* cudaStream_t as an integer (default 0) */
+    PS_OPT_STREAM = 3,                    /* cudaStream_t as an integer (default 0); only while nothing is pending.
+                                           * Work already enqueued on the old stream is ordered before the new one. */
     PS_OPT_QUEUE_GROUPS = 4,              /* max complete-but-unapplied groups (default 64) */
     PS_OPT_LOG_UPDATES = 5,               /* how many most recent updates the log keeps (default max(1024, 2^20 / c)) */
     PS_OPT_TIMING = 6,                    /* 1: bracket every update kernel with CUDA events (ps_kernel_time) */
     PS_OPT_KERNEL = 7,                    /* ps_kernel_choice (default PS_KERNEL_AUTO) */
-    PS_OPT_PROTOCOL = 10,                 /* ps_protocol (default PS_PROTOCOL_SOFTSYNC); only while nothing is pending */
+    PS_OPT_BLOCK_THREADS = 8,             /* threads per block: 128, 256 or 512; 0 = default (128; 256 for PS_KERNEL_BULK) */
     PS_OPT_OVERLAP_LAUNCH = 9,            /* 1: update kernels are launched as programmatic dependents (see below); default 0 */
-    PS_OPT_BLOCK_THREADS = 8              /* threads per block: 128, 256 or 512; 0 = default (128) */
+    PS_OPT_PROTOCOL = 10,                 /* ps_protocol (default PS_PROTOCOL_SOFTSYNC); only while nothing is pending */
+    PS_OPT_GROUP_SIZE = 11,               /* read-only: c = floor(lambda / n) of Eq. 2 */
+    PS_OPT_LAST_KERNEL = 12,              /* read-only: ps_kernel_choice the most recent update launch took (0: none yet) */
+    PS_OPT_LAUNCHES_SCALAR = 13,          /* read-only: update launches so far that took the scalar kernel, */
+    PS_OPT_LAUNCHES_VECTOR = 14,          /*            the vector kernel, */
+    PS_OPT_LAUNCHES_BULK = 15,            /*            the bulk-copy kernel */
+    PS_OPT_BULK_TILE = 16,                /* PS_KERNEL_BULK: elements per shared-memory tile, a power of two in
+                                           * [256, 8192] (halved until the stages of one block fit an SM's shared
+                                           * memory); 0 = chosen from the launch's gradient count (default) */
+    PS_OPT_BULK_STAGES = 17,              /* PS_KERNEL_BULK: tiles in flight per block, 2..8 (default 4) */
+    PS_OPT_BULK_WAIT_LIMIT = 18,          /* PS_KERNEL_BULK: polls of a copy barrier before the kernel gives up
+                                           * (default 2^22, about a second; at least 16) */
+    PS_OPT_BULK_SELFTEST = 19             /* PS_KERNEL_BULK, diagnostics: 1 makes block 0 of the NEXT launch announce 16
+                                           * bytes more than it copies for its first tile, so that tile's wait runs out;
+                                           * the launch then ends with PS_ERR_DEVICE_WAIT recorded.  Resets to 0. */
 };
 
 /* PS_OPT_OVERLAP_LAUNCH = 1 lets an update kernel start while the previous kernel on the stream is still
@@ -83,14 +102,26 @@ enum ps_option {
 enum ps_protocol { PS_PROTOCOL_SOFTSYNC = 0, PS_PROTOCOL_HARDSYNC = 1 };
 
 enum ps_kernel_choice {
-    PS_KERNEL_AUTO = 0,                   /* vector kernel when every pointer is 16-byte aligned, else scalar */
-    PS_KERNEL_SCALAR = 1,                 /* one element per thread and iteration */
-    PS_KERNEL_VECTOR = 2                  /* 16-byte loads and stores */
+    PS_KERNEL_AUTO = 0,                   /* vector kernel when the pointers are aligned for it, else scalar */
+    PS_KERNEL_SCALAR = 1,                 /* one element per thread */
+    PS_KERNEL_VECTOR = 2,                 /* four elements per thread, streamed through registers: 16-byte accesses to
+                                           * theta, v and fp32 gradients, 8-byte ones to bf16 gradients and the bf16
+                                           * mirror; needs exactly those alignments */
+    PS_KERNEL_BULK = 3                    /* persistent blocks that stage tiles of theta, v and the gradients in shared
+                                           * memory with bulk asynchronous copies (cp.async.bulk + mbarrier, one block per
+                                           * cluster, no multicast).  Needs every pointer 16-byte aligned and at most 16
+                                           * gradients per launch (T * c <= 16), else PS_ERR_INVALID_ARG.  Same bits as the
+                                           * other kernels.  Never chosen by PS_KERNEL_AUTO: on this element-wise, touch-once
+                                           * pass it measures slower than the register kernel; it exists so that the
+                                           * comparison can be repeated.  Every barrier wait in it is bounded
+                                           * (PS_OPT_BULK_WAIT_LIMIT).  Its first launch allocates 64 bytes of pinned host
+                                           * memory for the status record. */
 };
 
 #define PS_MAX_GROUP 256                  /* largest c = floor(lambda / n) */
 #define PS_MAX_FUSE_T 16                  /* largest temporal-fusion depth */
 #define PS_MAX_ENTRIES 512                /* largest T * c one kernel pass takes; T is clamped to fit */
+#define PS_MAX_LAYERS 64                  /* largest layer table of ps_set_layer_multipliers */
 
 /* One gradient's part in one weight update; what the server decided, for checking
  * against Section 2.1 (timestamp, staleness) and Eq. 2-3 (grouping, scale). */
@@ -99,10 +130,12 @@ typedef struct ps_log_entry {
     int64_t push_index;                   /* how many gradients this learner had pushed before */
     int64_t ts_grad;                      /* j: timestamp of the weights the gradient was computed on */
     int64_t tau;                          /* staleness i - j >= 0 */
-    int64_t sigma;                        /* staleness used in the learning rate, >= 1 */
+    int64_t sigma;                        /* staleness used in the learning rate: max(tau, 1) for PS_MOD_INV_STALENESS,
+                                           * 1 for PS_MOD_CONSTANT, tau for PS_MOD_EXP_STALENESS */
     int32_t learner;
     int32_t position;                     /* place in the summation order of the group, 0 .. c-1 */
-    float scale;                          /* s = alpha0 / (c * sigma), rounded to fp32 once */
+    float scale;                          /* s = alpha0 / (c * sigma) (alpha0 * rho^tau / c for the exponential penalty),
+                                           * rounded to fp32 once */
     float decay;                          /* d = weight_decay * sum of the group's scales (fp32) */
 } ps_log_entry;
 
@@ -117,16 +150,18 @@ int ps_create(ps_t **out, int64_t num_params, int lambda, int n,
 int ps_destroy(ps_t *ps);
 
 /* Binds caller-owned device buffers of num_params fp32 each: weights theta and momentum v.
- * They must stay valid until ps_destroy.  4-byte alignment is enough; 16-byte alignment
- * enables the vector kernel.  Does not touch their contents (a bf16 mirror bound earlier is refilled
- * from the new weights). */
+ * They must stay valid until ps_destroy and must not overlap.  4-byte alignment is enough; 16-byte
+ * alignment enables the vector kernel.  Does not touch their contents (a bf16 mirror bound earlier is
+ * refilled from the new weights). */
 int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev);
 
-/* Sets theta_0 (copied from w_src, host memory if src_is_host != 0, else device), zeroes the
- * momentum, resets the timestamp to 0 and drops pending gradients and the log. */
+/* The starting point of Section 2.1: sets theta_0 (copied from w_src, host memory if src_is_host != 0,
+ * else device), zeroes the momentum, resets the timestamp to 0 (the clock of Section 2.1 starts at
+ * 0 and gains one per weight update), and drops pending gradients, the log and a recorded
+ * PS_ERR_DEVICE_WAIT. */
 int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host);
 
-/* Binds a caller-owned device buffer of num_params bf16 values (2-byte aligned; 16-byte aligned keeps the
+/* Binds a caller-owned device buffer of num_params bf16 values (2-byte aligned; 8-byte aligned keeps the
  * vector kernel) that from now on always holds theta rounded to nearest-even bf16: it is filled at once
  * (and by ps_init_weights), and every ps_apply_update rewrites it in the same pass that updates theta
  * (2 more bytes per element instead of a separate conversion pass).  Learners that compute in bf16 can
@@ -146,8 +181,26 @@ int ps_get_option(ps_t *ps, int key, int64_t *value);
 
 /* Learning-rate schedule (Section 4.3 lowers alpha0 in steps during training): sets the base rate for
  * gradients pushed from now on.  Gradients already pushed keep the rate that was in force when they
- * arrived (Section 2.4 sets the rate "for an incoming gradient"). */
+ * arrived (the rate of Section 2.4, Eq. 3 is fixed per gradient as it comes in). */
 int ps_set_alpha0(ps_t *ps, float alpha0);
+
+/* Base rho of the exponential staleness penalty, alpha = alpha0 * rho^tau, used by PS_MOD_EXP_STALENESS
+ * (Section 1 discusses that rule as the earlier proposal and gives no formula; this form gives a fresh
+ * gradient, tau = 0, the full alpha0).  0 < rho <= 1, default 0.5; rho = 1 is the constant rate.  Only
+ * while no gradient is pending. */
+int ps_set_penalty_base(ps_t *ps, float rho);
+
+/* Per-layer multipliers.  The small network of Section 4.1 follows a Caffe model, in which every layer
+ * carries a learning-rate and a weight-decay multiplier (commonly 2 and 0 for biases).  Layer q covers
+ * elements [bounds_host[q], bounds_host[q+1]) with bounds_host[0] = 0, bounds_host[num_layers] = num_params,
+ * ascending; its elements are updated with
+ *     v = momentum * v + lr_mult[q] * (acc + (wd_mult[q] * d) * theta)
+ * (each product and sum rounded once), i.e. rate alpha * lr_mult[q] and decay weight_decay * wd_mult[q].
+ * Multipliers of 1 give exactly the bits of a server without a table.  num_layers = 0 removes the table;
+ * at most PS_MAX_LAYERS.  The three arrays are host memory and are copied.  Only while no gradient is
+ * pending. */
+int ps_set_layer_multipliers(ps_t *ps, int num_layers, const int64_t *bounds_host,
+                             const float *lr_mult_host, const float *wd_mult_host);
 
 /* pullWeights (Section 2.1): *ts receives the server timestamp i a gradient computed on these
  * weights must carry.  If out_dev != NULL, every complete pending group is applied first and
@@ -186,13 +239,26 @@ int ps_push_gradient_host(ps_t *ps, int learner, const void *grad_host, int64_t 
 
 /* Receive buffers for learners on the same GPU (the counterpart of the server-side receive buffer of the
  * paper's MPI transport, Section 2.3): ps_acquire_slot lends one free staging slot (bound with
- * ps_bind_staging); the learner writes its gradient there with its own kernels or copies, ordered before
- * the update on the server's stream, and hands it over with ps_push_slot, which behaves like
- * ps_push_gradient and returns the slot to the pool once the update that consumes it is enqueued.  A slot
- * that will not be pushed goes back with ps_release_slot.  PS_ERR_QUEUE_FULL when every slot is in use. */
+ * ps_bind_staging); the learner writes its gradient there with its own kernels or copies and hands it over
+ * with ps_push_slot, which behaves like ps_push_gradient and returns the slot to the pool once the update
+ * that consumes it is enqueued.  A slot that will not be pushed goes back with ps_release_slot.
+ * PS_ERR_QUEUE_FULL when every slot is in use.
+ *
+ * Two orderings are the learner's to keep, because a recycled slot may still be read by the update kernel
+ * that consumed its previous gradient, and the next update must not start before the new gradient is there:
+ *   (1) the write into the slot comes AFTER the slot's previous consumer: true for work enqueued on the
+ *       server's stream; a learner writing on another stream first calls ps_slot_wait(ps, id, its stream);
+ *   (2) the write comes BEFORE the update that consumes it: true for work enqueued on the server's stream
+ *       before ps_apply_update; a learner writing on another stream calls ps_slot_written(ps, id, its
+ *       stream) after enqueuing the write and before ps_push_slot, which makes the server's stream wait.
+ * A launch that consumes a gradient pushed with ps_push_slot is never started early by
+ * PS_OPT_OVERLAP_LAUNCH (its producer may be the kernel directly before it). */
 int ps_acquire_slot(ps_t *ps, void **slot_dev, int *slot_id);
 int ps_push_slot(ps_t *ps, int learner, int slot_id, int64_t ts);
 int ps_release_slot(ps_t *ps, int slot_id);
+/* stream: a cudaStream_t.  Both need a slot currently lent by ps_acquire_slot. */
+int ps_slot_wait(ps_t *ps, int slot_id, void *stream);      /* `stream` waits until the slot's last consumer has finished */
+int ps_slot_written(ps_t *ps, int slot_id, void *stream);   /* the server's stream waits for what `stream` holds so far */
 
 /* applyUpdate fused with sumGradients (Section 2.1; Eq. 2 with the learning rate of Eq. 3):
  * takes up to PS_OPT_FUSE_T complete groups, oldest first, and applies them in ONE kernel pass
@@ -207,19 +273,29 @@ int ps_release_slot(ps_t *ps, int slot_id);
  * PS_ERR_NOT_READY. */
 int ps_apply_update(ps_t *ps);
 
-/* Applies every complete pending group (repeated ps_apply_update).  Returns the number applied (>= 0). */
+/* Applies every complete pending group (repeated ps_apply_update: Section 2.1's applyUpdate for each group
+ * of Eq. 2 that is waiting).  Returns the number applied (>= 0). */
 int ps_flush(ps_t *ps);
 
-/* Blocks until everything this handle enqueued (main stream and read-back stream) has finished. */
+/* Blocks until everything this handle enqueued (main stream and read-back stream) has finished.
+ * Returns PS_ERR_DEVICE_WAIT if an update kernel has given up on a bounded wait since ps_init_weights. */
 int ps_synchronize(ps_t *ps);
 
-/* Copies the log entries of updates [first_update, first_update + count) to out_host
+/* Waits for the stream, then reports the status record of the bulk-copy kernel: *code 0 = no wait has run
+ * out; else 1, with the block, the block's tile counter and the stage whose copy barrier did not complete.
+ * Any output pointer may be NULL. */
+int ps_kernel_status(ps_t *ps, int *code, int *block, int64_t *tile, int *stage);
+
+/* The server's record of what Section 2.1 defines per gradient (its timestamp j, the server timestamp i it
+ * met, the staleness i - j: the quantity whose distribution Fig. 1 shows) and of Eq. 2-3 (group membership,
+ * summation order, scale).  Copies the entries of updates [first_update, first_update + count) to out_host
  * (count * c entries, update-major, in summation order). */
 int ps_get_update_log(ps_t *ps, int64_t first_update, int64_t count, ps_log_entry *out_host);
 
-/* Device pointers of the bound state and both clocks: ts_applied counts updates whose kernel has
- * been enqueued; ts_logical = ts_applied + complete pending groups (what ps_pull_weights returns).
- * Any output pointer may be NULL. */
+/* Device pointers of the bound state and both readings of the timestamp of Section 2.1: ts_applied
+ * counts updates whose kernel has been enqueued; ts_logical = ts_applied + complete pending groups (what
+ * ps_pull_weights returns: a complete group has already advanced the clock the learners see, whether or
+ * not its kernel has been launched).  Any output pointer may be NULL. */
 int ps_peek_state(ps_t *ps, const float **w_dev, const float **v_dev,
                   int64_t *ts_applied, int64_t *ts_logical);
 

@@ -19,18 +19,23 @@ import torch
 from . import build as _build
 
 # ---- constants mirrored from include/softsync_ps.h ---------------------------
-PS_MOD_CONSTANT, PS_MOD_INV_STALENESS = 0, 1
+PS_MOD_CONSTANT, PS_MOD_INV_STALENESS, PS_MOD_EXP_STALENESS = 0, 1, 2
 PS_OK, PS_READY = 0, 1
 PS_ERR_INVALID_ARG, PS_ERR_BAD_LEARNER, PS_ERR_BAD_TIMESTAMP, PS_ERR_NOT_READY = -1, -2, -3, -4
 PS_ERR_QUEUE_FULL, PS_ERR_CUDA, PS_ERR_NOMEM, PS_ERR_NO_STATE, PS_ERR_LOG_EVICTED, PS_ERR_BARRIER = -5, -6, -7, -8, -9, -10
+PS_ERR_DEVICE_WAIT = -11
 PS_GRAD_FP32, PS_GRAD_BF16 = 0, 1
 (PS_OPT_GRAD_DTYPE, PS_OPT_FUSE_T, PS_OPT_STREAM, PS_OPT_QUEUE_GROUPS, PS_OPT_LOG_UPDATES,
- PS_OPT_TIMING, PS_OPT_KERNEL, PS_OPT_BLOCK_THREADS, PS_OPT_OVERLAP_LAUNCH, PS_OPT_PROTOCOL) = range(1, 11)
+ PS_OPT_TIMING, PS_OPT_KERNEL, PS_OPT_BLOCK_THREADS, PS_OPT_OVERLAP_LAUNCH, PS_OPT_PROTOCOL,
+ PS_OPT_GROUP_SIZE, PS_OPT_LAST_KERNEL, PS_OPT_LAUNCHES_SCALAR, PS_OPT_LAUNCHES_VECTOR, PS_OPT_LAUNCHES_BULK,
+ PS_OPT_BULK_TILE, PS_OPT_BULK_STAGES, PS_OPT_BULK_WAIT_LIMIT, PS_OPT_BULK_SELFTEST) = range(1, 20)
 PS_PROTOCOL_SOFTSYNC, PS_PROTOCOL_HARDSYNC = 0, 1
-PS_KERNEL_AUTO, PS_KERNEL_SCALAR, PS_KERNEL_VECTOR = 0, 1, 2
-PS_MAX_GROUP, PS_MAX_FUSE_T, PS_MAX_ENTRIES = 256, 16, 512
+PS_KERNEL_AUTO, PS_KERNEL_SCALAR, PS_KERNEL_VECTOR, PS_KERNEL_BULK = 0, 1, 2, 3
+PS_MAX_GROUP, PS_MAX_FUSE_T, PS_MAX_ENTRIES, PS_MAX_LAYERS = 256, 16, 512, 64
 
-MODULATIONS = {"constant": PS_MOD_CONSTANT, "inv_staleness": PS_MOD_INV_STALENESS}
+MODULATIONS = {"constant": PS_MOD_CONSTANT, "inv_staleness": PS_MOD_INV_STALENESS, "exp_staleness": PS_MOD_EXP_STALENESS}
+KERNELS = {"auto": PS_KERNEL_AUTO, "scalar": PS_KERNEL_SCALAR, "vector": PS_KERNEL_VECTOR, "bulk": PS_KERNEL_BULK}
+TORCH_DTYPE = {"fp32": torch.float32, "bf16": torch.bfloat16}
 GRAD_DTYPES = {"fp32": PS_GRAD_FP32, "bf16": PS_GRAD_BF16}
 
 LOG_DTYPE = np.dtype([
@@ -41,7 +46,8 @@ LOG_DTYPE = np.dtype([
 EXPORTS = (
     "ps_create", "ps_destroy", "ps_bind_state", "ps_init_weights", "ps_bind_staging", "ps_bind_weight_mirror",
     "ps_pull_weights_bf16",
-    "ps_set_option", "ps_get_option", "ps_set_alpha0", "ps_pull_weights", "ps_pull_weights_host", "ps_pull_weights_host_async",
+    "ps_set_option", "ps_get_option", "ps_set_alpha0", "ps_set_penalty_base", "ps_set_layer_multipliers",
+    "ps_slot_wait", "ps_slot_written", "ps_kernel_status", "ps_pull_weights", "ps_pull_weights_host", "ps_pull_weights_host_async",
     "ps_push_gradient", "ps_push_gradient_host", "ps_acquire_slot", "ps_push_slot", "ps_release_slot", "ps_apply_update", "ps_flush", "ps_synchronize",
     "ps_get_update_log", "ps_peek_state", "ps_export_state", "ps_import_state", "ps_kernel_time", "ps_last_cuda_error", "ps_status_string",
 )
@@ -72,6 +78,11 @@ def _load() -> C.CDLL:
         "ps_set_option": [vp, i32, i64],
         "ps_get_option": [vp, i32, C.POINTER(i64)],
         "ps_set_alpha0": [vp, f32],
+        "ps_set_penalty_base": [vp, f32],
+        "ps_set_layer_multipliers": [vp, i32, vp, vp, vp],
+        "ps_slot_wait": [vp, i32, vp],
+        "ps_slot_written": [vp, i32, vp],
+        "ps_kernel_status": [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i64), C.POINTER(i32)],
         "ps_pull_weights": [vp, vp, C.POINTER(i64)],
         "ps_pull_weights_host": [vp, vp, C.POINTER(i64)],
         "ps_pull_weights_host_async": [vp, vp, C.POINTER(i64)],
@@ -112,6 +123,11 @@ ps_pull_weights_bf16 = lib.ps_pull_weights_bf16
 ps_set_option = lib.ps_set_option
 ps_get_option = lib.ps_get_option
 ps_set_alpha0 = lib.ps_set_alpha0
+ps_set_penalty_base = lib.ps_set_penalty_base
+ps_set_layer_multipliers = lib.ps_set_layer_multipliers
+ps_slot_wait = lib.ps_slot_wait
+ps_slot_written = lib.ps_slot_written
+ps_kernel_status = lib.ps_kernel_status
 ps_pull_weights = lib.ps_pull_weights
 ps_pull_weights_host = lib.ps_pull_weights_host
 ps_pull_weights_host_async = lib.ps_pull_weights_host_async
@@ -141,6 +157,26 @@ def _check(status: int, where: str) -> int:
     return status
 
 
+def require_tensor(t: torch.Tensor, dtype: torch.dtype, count: int, what: str, on_gpu: bool,
+                   device: Optional[torch.device] = None) -> None:
+    """The library sees only an address.  Refuse a tensor whose memory is not what a kernel or copy that
+    reads or writes `count` elements of `dtype` there will assume: wrong element type, too short, strided,
+    or (on_gpu) not on the server's GPU."""
+    if t.dtype != dtype:
+        raise TypeError("%s must be %s, got %s" % (what, dtype, t.dtype))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % what)
+    if t.numel() < count:
+        raise ValueError("%s holds %d elements, the server has %d parameters" % (what, t.numel(), count))
+    if on_gpu and count > 0:
+        if not t.is_cuda:
+            raise ValueError("%s must live on the server's GPU" % what)
+        if device is not None and t.device != device:
+            raise ValueError("%s is on %s, the server on %s" % (what, t.device, device))
+    if not on_gpu and t.is_cuda:
+        raise ValueError("%s must live in host memory" % what)
+
+
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
     return None if t is None else t.data_ptr()
 
@@ -160,7 +196,7 @@ class ParameterServer:
         self._h = C.c_void_p()
         self.num_params = int(num_params)
         self.num_learners = int(num_learners)
-        self.c = num_learners // n if n >= 1 else 0
+        self.c = 0                    # group size of Eq. 2, asked from the library once it exists
         self.grad_dtype = grad_dtype
         self._held = collections.deque()
         self._host_held = []          # pinned host gradients whose upload may still be in flight
@@ -173,6 +209,7 @@ class ParameterServer:
         with ctx:
             _check(ps_create(C.byref(self._h), num_params, num_learners, n, alpha0, momentum, weight_decay,
                              MODULATIONS[modulation]), "ps_create")
+        self.c = self.get_option(PS_OPT_GROUP_SIZE)
         if state is not None:
             self.bind_state(*state)
         elif allocate and num_params > 0:
@@ -199,14 +236,20 @@ class ParameterServer:
             pass
 
     # -- set-up ---------------------------------------------------------------
+    def _check_device_tensor(self, t: torch.Tensor, dtype: torch.dtype, what: str) -> None:
+        require_tensor(t, dtype, self.num_params, what, on_gpu=True, device=self.device)
+
     def bind_state(self, w: torch.Tensor, v: torch.Tensor) -> None:
-        assert w.dtype == torch.float32 and v.dtype == torch.float32
-        assert w.numel() >= self.num_params and v.numel() >= self.num_params
+        self._check_device_tensor(w, torch.float32, "weights")
+        self._check_device_tensor(v, torch.float32, "momentum")
         _check(ps_bind_state(self._h, w.data_ptr(), v.data_ptr()), "ps_bind_state")
         self.w, self.v = w, v
 
     def init_weights(self, w0: torch.Tensor) -> None:
-        assert w0.dtype == torch.float32 and w0.is_contiguous() and w0.numel() == self.num_params
+        if w0.is_cuda:
+            self._check_device_tensor(w0, torch.float32, "initial weights")
+        else:
+            self._check_host_tensor(w0, torch.float32, "initial weights")
         _check(ps_init_weights(self._h, w0.data_ptr(), 0 if w0.is_cuda else 1), "ps_init_weights")
         self._held.clear()
 
@@ -221,7 +264,7 @@ class ParameterServer:
         """Keep a bf16 copy of the weights current in `mirror` (allocated here if not given)."""
         if mirror is None:
             mirror = torch.empty(max(1, self.num_params), dtype=torch.bfloat16, device=self.device)
-        assert mirror.dtype == torch.bfloat16 and mirror.numel() >= self.num_params
+        self._check_device_tensor(mirror, torch.bfloat16, "weight mirror")
         _check(ps_bind_weight_mirror(self._h, mirror.data_ptr()), "ps_bind_weight_mirror")
         self.mirror = mirror
         return mirror
@@ -232,6 +275,23 @@ class ParameterServer:
     def set_alpha0(self, alpha0: float) -> None:
         """Base learning rate for gradients pushed from now on."""
         _check(ps_set_alpha0(self._h, alpha0), "ps_set_alpha0")
+
+    def set_penalty_base(self, rho: float) -> None:
+        """Base of the exponential staleness penalty alpha0 * rho**tau (modulation "exp_staleness")."""
+        _check(ps_set_penalty_base(self._h, rho), "ps_set_penalty_base")
+
+    def set_layer_multipliers(self, bounds, lr_mult, wd_mult) -> None:
+        """Layer q = elements [bounds[q], bounds[q+1]) with learning-rate and weight-decay multipliers;
+        empty lists remove the table."""
+        bounds = np.ascontiguousarray(bounds, dtype=np.int64)
+        lr_mult = np.ascontiguousarray(lr_mult, dtype=np.float32)
+        wd_mult = np.ascontiguousarray(wd_mult, dtype=np.float32)
+        n = int(lr_mult.size)
+        if n and (wd_mult.size != n or bounds.size != n + 1):
+            raise ValueError("need num_layers multipliers of each kind and num_layers + 1 bounds")
+        _check(ps_set_layer_multipliers(self._h, n, bounds.ctypes.data if n else None,
+                                        lr_mult.ctypes.data if n else None, wd_mult.ctypes.data if n else None),
+               "ps_set_layer_multipliers")
 
     def get_option(self, key: int) -> int:
         out = C.c_int64()
@@ -247,22 +307,24 @@ class ParameterServer:
         if out is None:
             _check(ps_pull_weights(self._h, None, C.byref(ts)), "ps_pull_weights")
             return ts.value
-        assert out.is_contiguous()
         applied_before = self.timestamps()[0]
         if out.dtype == torch.bfloat16:
-            assert out.is_cuda
+            self._check_device_tensor(out, torch.bfloat16, "bf16 pull target")
             _check(ps_pull_weights_bf16(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_bf16")
         elif out.is_cuda:
-            assert out.dtype == torch.float32
+            self._check_device_tensor(out, torch.float32, "pull target")
             _check(ps_pull_weights(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights")
-        elif non_blocking:
-            assert out.dtype == torch.float32
-            _check(ps_pull_weights_host_async(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host_async")
         else:
-            assert out.dtype == torch.float32
-            _check(ps_pull_weights_host(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host")
+            self._check_host_tensor(out, torch.float32, "host pull target")
+            if non_blocking:
+                _check(ps_pull_weights_host_async(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host_async")
+            else:
+                _check(ps_pull_weights_host(self._h, out.data_ptr(), C.byref(ts)), "ps_pull_weights_host")
         self._release(self.timestamps()[0] - applied_before)     # the pull applied every complete group first
         return ts.value
+
+    def _check_host_tensor(self, t: torch.Tensor, dtype: torch.dtype, what: str) -> None:
+        require_tensor(t, dtype, self.num_params, what, on_gpu=False)
 
     def _release(self, groups: int) -> None:
         """Drop the references to the gradients of `groups` applied groups (oldest first)."""
@@ -271,10 +333,13 @@ class ParameterServer:
 
     def push_gradient(self, learner: int, grad: torch.Tensor, ts: int) -> bool:
         """True if this push completed a group of c (an update can be applied)."""
+        want = TORCH_DTYPE[self.grad_dtype]
         if grad.is_cuda:
+            self._check_device_tensor(grad, want, "gradient")
             r = _check(ps_push_gradient(self._h, learner, grad.data_ptr(), ts), "ps_push_gradient")
             self._held.append(grad)
         else:
+            self._check_host_tensor(grad, want, "host gradient")
             r = _check(ps_push_gradient_host(self._h, learner, grad.data_ptr(), ts), "ps_push_gradient_host")
             self._held.append(None)
             self._host_held.append(grad)
@@ -296,6 +361,14 @@ class ParameterServer:
         r = _check(ps_push_slot(self._h, learner, slot_id, ts), "ps_push_slot")
         self._held.append(None)
         return r == PS_READY
+
+    def slot_wait(self, slot_id: int, stream: torch.cuda.Stream) -> None:
+        """Make `stream` wait until the update kernel that last read this (recycled) slot has finished."""
+        _check(ps_slot_wait(self._h, slot_id, stream.cuda_stream), "ps_slot_wait")
+
+    def slot_written(self, slot_id: int, stream: torch.cuda.Stream) -> None:
+        """Tell the server that the slot's gradient is produced by the work enqueued on `stream` so far."""
+        _check(ps_slot_written(self._h, slot_id, stream.cuda_stream), "ps_slot_written")
 
     def release_slot(self, slot_id: int) -> None:
         _check(ps_release_slot(self._h, slot_id), "ps_release_slot")
@@ -342,6 +415,12 @@ class ParameterServer:
     def staleness_histogram(self, first_update: int = 0) -> np.ndarray:
         """counts[t] = gradients applied with staleness t (the quantity of Fig. 1), from the held update log."""
         return np.bincount(self.update_log(first_update)["tau"])
+
+    def kernel_status(self):
+        """(code, block, tile, stage) of the bulk-copy kernel's status record; code 0 = no wait has run out."""
+        code, block, tile, stage = C.c_int(), C.c_int(), C.c_int64(), C.c_int()
+        _check(ps_kernel_status(self._h, C.byref(code), C.byref(block), C.byref(tile), C.byref(stage)), "ps_kernel_status")
+        return code.value, block.value, tile.value, stage.value
 
     def kernel_time(self) -> Tuple[float, int]:
         ms, n = C.c_double(), C.c_int64()

@@ -1,6 +1,7 @@
 """Build libsoftsync_ps.so (the C-ABI library with its sm_100a kernels) in-tree with nvcc."""
 from __future__ import annotations
 
+import hashlib
 import os
 import shutil
 import subprocess
@@ -23,11 +24,24 @@ def nvcc() -> str:
     return exe
 
 
+STAMP = LIB + ".hash"            # digest of the sources and flags the library was built from
+
+
+def source_digest() -> str:
+    h = hashlib.sha256(" ".join(NVCC_FLAGS).encode())
+    for path in [os.path.join(CSRC, s) for s in SOURCES] + HEADERS:
+        with open(path, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
 def is_stale() -> bool:
-    if not os.path.exists(LIB):
+    """True unless the library exists and was built from exactly the present sources (file times are not
+    trusted: a copied tree does not keep them)."""
+    if not os.path.exists(LIB) or not os.path.exists(STAMP):
         return True
-    deps = [os.path.join(CSRC, s) for s in SOURCES] + HEADERS
-    return any(os.path.getmtime(d) > os.path.getmtime(LIB) for d in deps)
+    with open(STAMP) as f:
+        return f.read().strip() != source_digest()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -35,20 +49,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     cmd = [nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
           ["-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+    if os.path.exists(STAMP):
+        os.remove(STAMP)
     subprocess.run(cmd, check=True)
+    with open(STAMP, "w") as f:
+        f.write(source_digest() + "\n")
     return LIB
 
 
 def ensure_built() -> str:
-    """Build the library if it is missing or older than its sources.  A stale library is kept when the
-    rebuild fails (no compiler on this machine); a missing one is an error."""
-    if not os.path.exists(LIB):
-        return build(force=True)
+    """Build the library if it is missing or was built from other sources.  A failed rebuild raises: a
+    library that does not match the header and the binding must not be loaded."""
     if is_stale():
-        try:
-            return build(force=True)
-        except Exception:
-            return LIB
+        return build(force=True)
     return LIB
 
 

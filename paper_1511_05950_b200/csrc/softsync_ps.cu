@@ -7,6 +7,7 @@
 #include "update_kernels.cuh"
 
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <deque>
 #include <mutex>
@@ -16,6 +17,8 @@
 
 namespace {
 
+using softsync::BulkPlan;
+using softsync::BulkStatus;
 using softsync::GradBf16;
 using softsync::GradFp32;
 using softsync::LaunchParams;
@@ -26,6 +29,7 @@ struct Entry {                 // one pushed gradient waiting for its update
     float alpha0;              // base rate in force when the gradient arrived
     const void *grad;
     int slot;                  // staging slot it occupies, -1 if borrowed from the caller
+    bool by_learner;           // the slot was lent to a learner (ps_push_slot): its producer may be a kernel
 };
 
 struct TimedLaunch { cudaEvent_t start, stop; };
@@ -37,7 +41,12 @@ struct ps_ctx {
     int64_t n = 0;
     int lambda = 0, split = 0, c = 0, modulation = 0;
     float alpha0 = 0, momentum = 0, weight_decay = 0;
+    float penalty_base = 0.5f;             // rho of PS_MOD_EXP_STALENESS
     int device = 0;
+
+    int num_layers = 0;                    // per-layer multipliers (0: none)
+    int64_t layer_end[PS_MAX_LAYERS] = {};
+    float layer_lr[PS_MAX_LAYERS] = {}, layer_wd[PS_MAX_LAYERS] = {};
 
     float *w = nullptr, *v = nullptr;
     unsigned short *mirror = nullptr;      // optional caller-owned bf16 copy of theta
@@ -45,6 +54,9 @@ struct ps_ctx {
     int64_t slot_bytes = 0;
     std::vector<int> free_slots;
     std::vector<char> slot_lent;           // 1 while a learner holds the slot between acquire and push
+    std::vector<cudaEvent_t> slot_consumed;  // recorded behind the update kernel that read the slot last (lazily created)
+    std::vector<char> slot_has_consumer;
+    std::vector<cudaEvent_t> slot_filled;    // recorded on a learner's stream by ps_slot_written (lazily created)
     int num_slots = 0;
 
     int grad_dtype = PS_GRAD_FP32;
@@ -56,8 +68,14 @@ struct ps_ctx {
     int protocol = PS_PROTOCOL_SOFTSYNC;
     int sm_count = 0;
 
+    int bulk_tile = 0, bulk_stages = 4, bulk_wait_limit = 1 << 20, bulk_selftest = 0;
+    BulkStatus *bulk_status = nullptr;     // pinned, device-mapped host memory (allocated by the first bulk launch)
+    bool bulk_attr_set[2][2] = {};         // dynamic shared-memory opt-in done, per (dtype, layers) instantiation
+
     int64_t ts_applied = 0;                // updates whose kernel has been enqueued
     int64_t launches = 0;                  // update kernels enqueued so far
+    int last_kernel = 0;                   // ps_kernel_choice of the most recent launch
+    int64_t launches_by_kind[4] = {};      // indexed by ps_kernel_choice
     std::deque<std::vector<Entry>> ready;  // complete groups, oldest first
     std::vector<Entry> filling;            // the group being collected (< c entries)
     std::vector<int64_t> push_count;       // per learner
@@ -127,9 +145,13 @@ bool entry_before(const Entry &a, const Entry &b)
 
 constexpr int kChunk = 8;            // gradient loads in flight per thread beyond the first EC
 constexpr int kHead = 16;            // largest compile-time first chunk of gradient loads
+constexpr int kBulkThreads = 256;
 
-template <typename GT, int VEC, int EC, bool MORE, int MAXE>
-cudaError_t launch_variant(const LaunchParams<MAXE> &p, int blocks, int threads, cudaStream_t stream)
+template <bool LAYERS> constexpr int seg_capacity() { return LAYERS ? PS_MAX_LAYERS : 1; }
+template <int MAXE, bool LAYERS> using Params = LaunchParams<MAXE, seg_capacity<LAYERS>()>;
+
+template <typename GT, int VEC, int EC, bool MORE, bool LAYERS, int MAXE>
+cudaError_t launch_variant(const Params<MAXE, LAYERS> &p, int blocks, int threads, cudaStream_t stream)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(blocks));
@@ -140,61 +162,143 @@ cudaError_t launch_variant(const LaunchParams<MAXE> &p, int blocks, int threads,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = p.overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, softsync::softsync_update_kernel<GT, VEC, EC, MORE, kChunk, MAXE>, p);
+    return cudaLaunchKernelEx(&cfg, softsync::softsync_update_kernel<GT, VEC, EC, MORE, kChunk, LAYERS, MAXE, seg_capacity<LAYERS>()>, p);
 }
 
 // E = T*c <= HEAD: the straight-line instantiation with exactly E loads up front.
-template <typename GT, int VEC, int HEAD, int MAXE, int EC = HEAD>
-cudaError_t launch_exact(int E, const LaunchParams<MAXE> &p, int blocks, int threads, cudaStream_t stream)
+template <typename GT, int VEC, int HEAD, bool LAYERS, int MAXE, int EC = HEAD>
+cudaError_t launch_exact(int E, const Params<MAXE, LAYERS> &p, int blocks, int threads, cudaStream_t stream)
 {
     if constexpr (EC == 0) {
         return cudaErrorInvalidValue;
     } else {
-        if (E == EC) return launch_variant<GT, VEC, EC, false, MAXE>(p, blocks, threads, stream);
-        return launch_exact<GT, VEC, HEAD, MAXE, EC - 1>(E, p, blocks, threads, stream);
+        if (E == EC) return launch_variant<GT, VEC, EC, false, LAYERS, MAXE>(p, blocks, threads, stream);
+        return launch_exact<GT, VEC, HEAD, LAYERS, MAXE, EC - 1>(E, p, blocks, threads, stream);
     }
 }
 
-template <typename GT, int VEC, int HEAD, int MAXE>
-cudaError_t launch_vector(int E, const LaunchParams<MAXE> &p, int blocks, int threads, cudaStream_t stream)
+template <typename GT, int VEC, int HEAD, bool LAYERS, int MAXE>
+cudaError_t launch_vector(int E, const Params<MAXE, LAYERS> &p, int blocks, int threads, cudaStream_t stream)
 {
     if constexpr (MAXE <= HEAD) {                        // the small parameter block: T*c <= HEAD always
-        return launch_exact<GT, VEC, MAXE, MAXE>(E, p, blocks, threads, stream);
+        return launch_exact<GT, VEC, MAXE, LAYERS, MAXE>(E, p, blocks, threads, stream);
     } else {
         if (E <= HEAD) return cudaErrorInvalidValue;     // such launches use the small parameter block
     }
-    return launch_variant<GT, VEC, HEAD, true, MAXE>(p, blocks, threads, stream);   // HEAD loads, then chunks
+    return launch_variant<GT, VEC, HEAD, true, LAYERS, MAXE>(p, blocks, threads, stream);   // HEAD loads, then chunks
 }
 
-template <int MAXE>
-cudaError_t launch_update(ps_ctx *ps, const LaunchParams<MAXE> &p, bool vector_ok)
+// The bulk-copy kernel: tile and grid sizes from the shared memory one block may take.
+template <typename GT, bool LAYERS, int MAXE>
+cudaError_t launch_bulk(ps_ctx *ps, const Params<MAXE, LAYERS> &p)
+{
+    constexpr int kSeg = seg_capacity<LAYERS>();
+    const int gb = ps->grad_dtype == PS_GRAD_BF16 ? 2 : 4;
+    const int E = p.T * p.c;
+    const size_t per_elem = 8 + static_cast<size_t>(E) * gb;
+    const int stages = ps->bulk_stages;
+    const size_t budget = 100 * 1024;                    // two blocks per SM
+    // default: the largest tile that leaves room for two blocks per SM; a tile asked for by option is
+    // halved until one block's stages fit the shared memory of an SM
+    int tile = ps->bulk_tile ? ps->bulk_tile : 8192;
+    const size_t limit = ps->bulk_tile ? 200 * 1024 : budget;
+    while (tile > 256 && static_cast<size_t>(stages) * tile * per_elem > limit) tile >>= 1;
+    const size_t smem = static_cast<size_t>(stages) * tile * per_elem;
+    if (smem > 220 * 1024) return cudaErrorInvalidConfiguration;
+    auto kernel = softsync::softsync_update_bulk_kernel<GT, LAYERS, MAXE, kSeg>;
+    bool &attr_set = ps->bulk_attr_set[gb == 2][LAYERS];
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    if (!ps->bulk_status) {
+        cudaError_t e = cudaHostAlloc(reinterpret_cast<void **>(&ps->bulk_status), 64, cudaHostAllocMapped);
+        if (e != cudaSuccess) return e;
+        std::memset(ps->bulk_status, 0, 64);
+    }
+    BulkPlan plan;
+    plan.tile_elems = tile;
+    plan.ntiles = p.n / tile;
+    plan.stages = stages;
+    plan.wait_limit = ps->bulk_wait_limit;
+    plan.selftest = ps->bulk_selftest;
+    ps->bulk_selftest = 0;
+    cudaError_t e = cudaHostGetDevicePointer(reinterpret_cast<void **>(&plan.status), ps->bulk_status, 0);
+    if (e != cudaSuccess) return e;
+    const int threads = ps->block_threads ? ps->block_threads : kBulkThreads;
+    const size_t per_sm = 227 * 1024;
+    const int by_smem = static_cast<int>(std::max<size_t>(1, per_sm / (smem + 1024)));
+    const int per_sm_blocks = std::max(1, std::min(by_smem, 2048 / threads));
+    const long long cap = static_cast<long long>(ps->sm_count) * per_sm_blocks;
+    const int blocks = static_cast<int>(std::max<long long>(1, std::min<long long>(plan.ntiles, cap)));
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+    cfg.blockDim = dim3(static_cast<unsigned>(threads));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = ps->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, p, plan);
+}
+
+enum LaunchKind { kScalar = PS_KERNEL_SCALAR, kVector = PS_KERNEL_VECTOR, kBulk = PS_KERNEL_BULK };
+
+template <int MAXE, bool LAYERS>
+cudaError_t launch_update(ps_ctx *ps, const Params<MAXE, LAYERS> &p, int kind)
 {
     const bool bf16 = ps->grad_dtype == PS_GRAD_BF16;
-    const int vec = vector_ok ? 4 : 1;
+    if (kind == kBulk) {
+        if constexpr (MAXE <= kHead) {
+            return bf16 ? launch_bulk<GradBf16, LAYERS, MAXE>(ps, p) : launch_bulk<GradFp32, LAYERS, MAXE>(ps, p);
+        } else {
+            return cudaErrorInvalidValue;                // checked by the caller: T*c <= 16 only
+        }
+    }
+    const int vec = kind == kVector ? 4 : 1;
     const int threads = ps->block_threads ? ps->block_threads : 128;
     const long long frags = std::max<long long>(1, (p.n + vec - 1) / vec);
     const long long blocks = (frags + threads - 1) / threads;    // one fragment per thread
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     const int b = static_cast<int>(blocks);
     const int E = p.T * p.c;
-    if (!vector_ok)
-        return bf16 ? launch_variant<GradBf16, 1, 0, true, MAXE>(p, b, threads, ps->stream)
-                    : launch_variant<GradFp32, 1, 0, true, MAXE>(p, b, threads, ps->stream);
-    return bf16 ? launch_vector<GradBf16, 4, kHead, MAXE>(E, p, b, threads, ps->stream)
-                : launch_vector<GradFp32, 4, kHead, MAXE>(E, p, b, threads, ps->stream);
+    if (kind == kScalar)
+        return bf16 ? launch_variant<GradBf16, 1, 0, true, LAYERS, MAXE>(p, b, threads, ps->stream)
+                    : launch_variant<GradFp32, 1, 0, true, LAYERS, MAXE>(p, b, threads, ps->stream);
+    return bf16 ? launch_vector<GradBf16, 4, kHead, LAYERS, MAXE>(E, p, b, threads, ps->stream)
+                : launch_vector<GradFp32, 4, kHead, LAYERS, MAXE>(E, p, b, threads, ps->stream);
 }
 
+bool aligned_to(const void *p, uintptr_t bytes) { return (reinterpret_cast<uintptr_t>(p) & (bytes - 1)) == 0; }
+
 // Fills the scale table of one launch (Eq. 3 folded with the 1/c of Eq. 2) for the `T`
-// oldest complete groups and the log entries that describe them.
-template <int MAXE>
-void build_launch(ps_ctx *ps, int T, LaunchParams<MAXE> &p, std::vector<ps_log_entry> &entries, bool &vector_ok)
+// oldest complete groups and the log entries that describe them.  vector_ok / bulk_ok: whether every
+// pointer of the launch is aligned for the widths those kernels use.
+template <int MAXE, bool LAYERS>
+void build_launch(ps_ctx *ps, int T, Params<MAXE, LAYERS> &p, std::vector<ps_log_entry> &entries,
+                  bool &vector_ok, bool &bulk_ok)
 {
     p.w = ps->w; p.v = ps->v; p.n = ps->n;
     p.momentum = ps->momentum; p.T = T; p.c = ps->c;
     p.overlap = ps->overlap_launch;
     p.reverse = static_cast<int>(ps->launches & 1);      // zig-zag over the vector from launch to launch
     p.mirror = ps->mirror;
-    vector_ok = aligned16(ps->w) && aligned16(ps->v) && aligned16(ps->mirror);
+    p.layers.count = 0;
+    if constexpr (LAYERS) {
+        p.layers.count = ps->num_layers;
+        for (int q = 0; q < ps->num_layers; ++q) {
+            p.layers.end[q] = ps->layer_end[q]; p.layers.lm[q] = ps->layer_lr[q]; p.layers.dm[q] = ps->layer_wd[q];
+        }
+    }
+    // the vector kernel moves theta and v in 16-byte pieces, fp32 gradients too; bf16 gradients and the
+    // bf16 mirror in 8-byte pieces.  The bulk copies need 16 bytes everywhere.
+    const uintptr_t grad_align = ps->grad_dtype == PS_GRAD_BF16 ? 8 : 16;
+    vector_ok = aligned16(ps->w) && aligned16(ps->v) && aligned_to(ps->mirror, 8);
+    bulk_ok = aligned16(ps->w) && aligned16(ps->v) && aligned_to(ps->mirror, 8);
     const double wd = static_cast<double>(ps->weight_decay);
     for (int t = 0; t < T; ++t) {
         std::vector<Entry> &grp = ps->ready[t];
@@ -202,11 +306,18 @@ void build_launch(ps_ctx *ps, int T, LaunchParams<MAXE> &p, std::vector<ps_log_e
         double sum = 0.0;
         for (int l = 0; l < ps->c; ++l) {
             const Entry &en = grp[l];
-            const float s = static_cast<float>(static_cast<double>(en.alpha0) /
-                                               (static_cast<double>(ps->c) * static_cast<double>(en.sigma)));
+            double step;
+            if (ps->modulation == PS_MOD_EXP_STALENESS)      // alpha0 * rho^tau, then the 1/c of Eq. 2
+                step = static_cast<double>(en.alpha0) * std::pow(static_cast<double>(ps->penalty_base), static_cast<double>(en.tau)) /
+                       static_cast<double>(ps->c);
+            else                                             // Eq. 3 (sigma = 1 for the constant rate)
+                step = static_cast<double>(en.alpha0) / (static_cast<double>(ps->c) * static_cast<double>(en.sigma));
+            const float s = static_cast<float>(step);
             p.s[t * ps->c + l] = s;
             p.g[t * ps->c + l] = en.grad;
-            vector_ok = vector_ok && aligned16(en.grad);
+            vector_ok = vector_ok && aligned_to(en.grad, grad_align);
+            bulk_ok = bulk_ok && aligned16(en.grad);
+            if (en.by_learner) p.overlap = 0;               // its producer may be the kernel directly before this one
             sum += static_cast<double>(s);
         }
         const float d = static_cast<float>(wd * sum);   // every gradient carries + wd * theta
@@ -253,16 +364,21 @@ int take_events(ps_ctx *ps, TimedLaunch &tl)
     return PS_OK;
 }
 
-template <int MAXE>
+template <int MAXE, bool LAYERS>
 int apply_groups(ps_ctx *ps, int T)
 {
-    LaunchParams<MAXE> p;
+    Params<MAXE, LAYERS> p;
     std::vector<ps_log_entry> entries;
     entries.reserve(static_cast<size_t>(T) * ps->c);
-    bool vector_ok = false;
-    build_launch<MAXE>(ps, T, p, entries, vector_ok);
-    if (ps->kernel_choice == PS_KERNEL_SCALAR) vector_ok = false;
+    bool vector_ok = false, bulk_ok = false;
+    build_launch<MAXE, LAYERS>(ps, T, p, entries, vector_ok, bulk_ok);
+    int kind = vector_ok ? kVector : kScalar;
+    if (ps->kernel_choice == PS_KERNEL_SCALAR) kind = kScalar;
     if (ps->kernel_choice == PS_KERNEL_VECTOR && !vector_ok) return PS_ERR_INVALID_ARG;
+    if (ps->kernel_choice == PS_KERNEL_BULK) {
+        if (!bulk_ok || T * ps->c > kHead) return PS_ERR_INVALID_ARG;
+        kind = kBulk;
+    }
 
     if (ps->n > 0) {
         const int rb = order_after_readback(ps);
@@ -274,11 +390,22 @@ int apply_groups(ps_ctx *ps, int T)
             if (rc != PS_OK) return rc;
             PS_CUDA(ps, cudaEventRecord(tl.start, ps->stream));
         }
-        PS_CUDA(ps, launch_update<MAXE>(ps, p, vector_ok));
+        PS_CUDA(ps, (launch_update<MAXE, LAYERS>(ps, p, kind)));
         if (timed) {
             PS_CUDA(ps, cudaEventRecord(tl.stop, ps->stream));
             ps->timed.push_back(tl);
         }
+        // a recycled slot may be handed out while this kernel still reads it: remember where the kernel ends
+        for (int t = 0; t < T; ++t)
+            for (const Entry &en : ps->ready[t])
+                if (en.slot >= 0) {
+                    if (!ps->slot_consumed[en.slot])
+                        PS_CUDA(ps, cudaEventCreateWithFlags(&ps->slot_consumed[en.slot], cudaEventDisableTiming));
+                    PS_CUDA(ps, cudaEventRecord(ps->slot_consumed[en.slot], ps->stream));
+                    ps->slot_has_consumer[en.slot] = 1;
+                }
+        ps->last_kernel = kind;
+        ps->launches_by_kind[kind] += 1;
     }
     ps->launches += 1;
     // the launch is enqueued: advance the clock, release slots, publish the log
@@ -304,10 +431,13 @@ int apply_some(ps_ctx *ps)
     if (ps->ready.empty()) return PS_ERR_NOT_READY;
     int T = static_cast<int>(std::min<int64_t>(ps->fuse_t, static_cast<int64_t>(ps->ready.size())));
     T = std::min(T, std::max(1, PS_MAX_ENTRIES / ps->c));
-    return T * ps->c <= 16 ? apply_groups<16>(ps, T) : apply_groups<PS_MAX_ENTRIES>(ps, T);
+    const bool small = T * ps->c <= kHead;
+    if (ps->num_layers > 0)
+        return small ? apply_groups<kHead, true>(ps, T) : apply_groups<PS_MAX_ENTRIES, true>(ps, T);
+    return small ? apply_groups<kHead, false>(ps, T) : apply_groups<PS_MAX_ENTRIES, false>(ps, T);
 }
 
-int push_common(ps_ctx *ps, int learner, const void *grad_dev, int64_t ts, int slot)
+int push_common(ps_ctx *ps, int learner, const void *grad_dev, int64_t ts, int slot, bool by_learner = false)
 {
     const int64_t i = ts_logical(ps);
     Entry en;
@@ -315,10 +445,13 @@ int push_common(ps_ctx *ps, int learner, const void *grad_dev, int64_t ts, int s
     en.push_index = ps->push_count[learner];
     en.ts_grad = ts;
     en.tau = i - ts;                                      // staleness (Section 2.1)
-    en.sigma = ps->modulation == PS_MOD_INV_STALENESS ? std::max<int64_t>(en.tau, 1) : 1;
+    en.sigma = 1;                                         // constant rate
+    if (ps->modulation == PS_MOD_INV_STALENESS) en.sigma = std::max<int64_t>(en.tau, 1);   // Eq. 3; alpha0 at tau = 0
+    if (ps->modulation == PS_MOD_EXP_STALENESS) en.sigma = en.tau;                          // the penalty's exponent
     en.alpha0 = ps->alpha0;
     en.grad = grad_dev;
     en.slot = slot;
+    en.by_learner = by_learner;
     ps->push_count[learner] += 1;
     ps->filling.push_back(en);
     if (static_cast<int>(ps->filling.size()) == ps->c) {  // group of c complete: the clock moves on
@@ -361,7 +494,7 @@ int ps_create(ps_t **out, int64_t num_params, int lambda, int n,
         if (!out) return PS_ERR_INVALID_ARG;
         *out = nullptr;
         if (num_params < 0 || lambda < 1 || n < 1 || n > lambda) return PS_ERR_INVALID_ARG;
-        if (modulation != PS_MOD_CONSTANT && modulation != PS_MOD_INV_STALENESS) return PS_ERR_INVALID_ARG;
+        if (modulation < PS_MOD_CONSTANT || modulation > PS_MOD_EXP_STALENESS) return PS_ERR_INVALID_ARG;
         if (lambda / n > PS_MAX_GROUP) return PS_ERR_INVALID_ARG;
         if (!(alpha0 == alpha0) || !(momentum == momentum) || !(weight_decay == weight_decay)) return PS_ERR_INVALID_ARG;
         ps_ctx *ps = new (std::nothrow) ps_ctx;
@@ -408,6 +541,9 @@ int ps_destroy(ps_t *ps)
         }
         release_events(ps);
         for (auto &tl : ps->spare_events) { cudaEventDestroy(tl.start); cudaEventDestroy(tl.stop); }
+        for (cudaEvent_t ev : ps->slot_consumed) if (ev) cudaEventDestroy(ev);
+        for (cudaEvent_t ev : ps->slot_filled) if (ev) cudaEventDestroy(ev);
+        if (ps->bulk_status) cudaFreeHost(ps->bulk_status);
         delete ps;
         return PS_OK;
     } PS_CATCH_ALL
@@ -418,6 +554,11 @@ int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev)
     try {
         if (!is_live(ps) || !w_dev || !v_dev || w_dev == v_dev) return PS_ERR_INVALID_ARG;
         if ((reinterpret_cast<uintptr_t>(w_dev) & 3u) || (reinterpret_cast<uintptr_t>(v_dev) & 3u)) return PS_ERR_INVALID_ARG;
+        {
+            const uintptr_t a = reinterpret_cast<uintptr_t>(w_dev), b = reinterpret_cast<uintptr_t>(v_dev);
+            const uintptr_t bytes = static_cast<uintptr_t>(ps->n) * sizeof(float);
+            if ((a < b ? b - a : a - b) < bytes) return PS_ERR_INVALID_ARG;          // the two ranges overlap
+        }
         if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
         if (w_dev == reinterpret_cast<float *>(ps->mirror) || v_dev == reinterpret_cast<float *>(ps->mirror))
             return PS_ERR_INVALID_ARG;
@@ -449,6 +590,10 @@ int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host)
         std::fill(ps->push_count.begin(), ps->push_count.end(), 0);
         ps->ts_applied = 0;
         ps->log.clear(); ps->log_first_update = 0;
+        if (ps->bulk_status && ps->bulk_status->code != 0) {
+            PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+            std::memset(ps->bulk_status, 0, sizeof(BulkStatus));
+        }
         return PS_OK;
     } PS_CATCH_ALL
 }
@@ -478,6 +623,12 @@ int ps_bind_staging(ps_t *ps, void *slots_dev, int64_t slot_bytes, int num_slots
         ps->free_slots.clear();
         for (int s = num_slots - 1; s >= 0; --s) ps->free_slots.push_back(s);
         ps->slot_lent.assign(num_slots, 0);
+        DeviceGuard on_device(ps);
+        for (cudaEvent_t ev : ps->slot_consumed) if (ev) cudaEventDestroy(ev);
+        for (cudaEvent_t ev : ps->slot_filled) if (ev) cudaEventDestroy(ev);
+        ps->slot_consumed.assign(num_slots, nullptr);
+        ps->slot_filled.assign(num_slots, nullptr);
+        ps->slot_has_consumer.assign(num_slots, 0);
         return PS_OK;
     } PS_CATCH_ALL
 }
@@ -495,9 +646,21 @@ int ps_set_option(ps_t *ps, int key, int64_t value)
         case PS_OPT_FUSE_T:
             if (value < 1 || value > PS_MAX_FUSE_T) return PS_ERR_INVALID_ARG;
             ps->fuse_t = static_cast<int>(value); return PS_OK;
-        case PS_OPT_STREAM:
+        case PS_OPT_STREAM: {
             if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
-            ps->stream = reinterpret_cast<cudaStream_t>(static_cast<uintptr_t>(value)); return PS_OK;
+            cudaStream_t next = reinterpret_cast<cudaStream_t>(static_cast<uintptr_t>(value));
+            if (next != ps->stream && ps->device >= 0 && ps->launches > 0) {
+                // updates and copies already enqueued on the old stream come first
+                DeviceGuard on_device(ps);
+                cudaEvent_t ev;
+                PS_CUDA(ps, cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+                cudaError_t e = cudaEventRecord(ev, ps->stream);
+                if (e == cudaSuccess) e = cudaStreamWaitEvent(next, ev, 0);
+                cudaEventDestroy(ev);
+                if (e != cudaSuccess) return cuda_fail(ps, e);
+            }
+            ps->stream = next; return PS_OK;
+        }
         case PS_OPT_QUEUE_GROUPS:
             if (value < 1) return PS_ERR_INVALID_ARG;
             ps->queue_groups = value; return PS_OK;
@@ -508,8 +671,20 @@ int ps_set_option(ps_t *ps, int key, int64_t value)
             if (value != 0 && value != 1) return PS_ERR_INVALID_ARG;
             ps->timing = static_cast<int>(value); return PS_OK;
         case PS_OPT_KERNEL:
-            if (value < PS_KERNEL_AUTO || value > PS_KERNEL_VECTOR) return PS_ERR_INVALID_ARG;
+            if (value < PS_KERNEL_AUTO || value > PS_KERNEL_BULK) return PS_ERR_INVALID_ARG;
             ps->kernel_choice = static_cast<int>(value); return PS_OK;
+        case PS_OPT_BULK_TILE:
+            if (value != 0 && (value < 256 || value > 8192 || (value & (value - 1)))) return PS_ERR_INVALID_ARG;
+            ps->bulk_tile = static_cast<int>(value); return PS_OK;
+        case PS_OPT_BULK_STAGES:
+            if (value < 2 || value > softsync::kBulkMaxStages) return PS_ERR_INVALID_ARG;
+            ps->bulk_stages = static_cast<int>(value); return PS_OK;
+        case PS_OPT_BULK_WAIT_LIMIT:
+            if (value < 16 || value > (int64_t{1} << 30)) return PS_ERR_INVALID_ARG;
+            ps->bulk_wait_limit = static_cast<int>(value); return PS_OK;
+        case PS_OPT_BULK_SELFTEST:
+            if (value != 0 && value != 1) return PS_ERR_INVALID_ARG;
+            ps->bulk_selftest = static_cast<int>(value); return PS_OK;
         case PS_OPT_PROTOCOL:
             if (value != PS_PROTOCOL_SOFTSYNC && value != PS_PROTOCOL_HARDSYNC) return PS_ERR_INVALID_ARG;
             if (value == PS_PROTOCOL_HARDSYNC && ps->split != 1) return PS_ERR_INVALID_ARG;
@@ -542,6 +717,15 @@ int ps_get_option(ps_t *ps, int key, int64_t *value)
         case PS_OPT_BLOCK_THREADS: *value = ps->block_threads; return PS_OK;
         case PS_OPT_OVERLAP_LAUNCH: *value = ps->overlap_launch; return PS_OK;
         case PS_OPT_PROTOCOL: *value = ps->protocol; return PS_OK;
+        case PS_OPT_GROUP_SIZE: *value = ps->c; return PS_OK;
+        case PS_OPT_LAST_KERNEL: *value = ps->last_kernel; return PS_OK;
+        case PS_OPT_LAUNCHES_SCALAR: *value = ps->launches_by_kind[PS_KERNEL_SCALAR]; return PS_OK;
+        case PS_OPT_LAUNCHES_VECTOR: *value = ps->launches_by_kind[PS_KERNEL_VECTOR]; return PS_OK;
+        case PS_OPT_LAUNCHES_BULK: *value = ps->launches_by_kind[PS_KERNEL_BULK]; return PS_OK;
+        case PS_OPT_BULK_TILE: *value = ps->bulk_tile; return PS_OK;
+        case PS_OPT_BULK_STAGES: *value = ps->bulk_stages; return PS_OK;
+        case PS_OPT_BULK_WAIT_LIMIT: *value = ps->bulk_wait_limit; return PS_OK;
+        case PS_OPT_BULK_SELFTEST: *value = ps->bulk_selftest; return PS_OK;
         default: return PS_ERR_INVALID_ARG;
         }
     } PS_CATCH_ALL
@@ -552,6 +736,36 @@ int ps_set_alpha0(ps_t *ps, float alpha0)
     try {
         if (!is_live(ps) || !(alpha0 == alpha0)) return PS_ERR_INVALID_ARG;
         ps->alpha0 = alpha0;
+        return PS_OK;
+    } PS_CATCH_ALL
+}
+
+int ps_set_penalty_base(ps_t *ps, float rho)
+{
+    try {
+        if (!is_live(ps) || !(rho > 0.0f) || rho > 1.0f) return PS_ERR_INVALID_ARG;
+        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+        ps->penalty_base = rho;
+        return PS_OK;
+    } PS_CATCH_ALL
+}
+
+int ps_set_layer_multipliers(ps_t *ps, int num_layers, const int64_t *bounds, const float *lr_mult, const float *wd_mult)
+{
+    try {
+        if (!is_live(ps) || num_layers < 0 || num_layers > PS_MAX_LAYERS) return PS_ERR_INVALID_ARG;
+        if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
+        if (num_layers == 0) { ps->num_layers = 0; return PS_OK; }
+        if (!bounds || !lr_mult || !wd_mult) return PS_ERR_INVALID_ARG;
+        if (bounds[0] != 0 || bounds[num_layers] != ps->n) return PS_ERR_INVALID_ARG;
+        for (int q = 0; q < num_layers; ++q) {
+            if (bounds[q] > bounds[q + 1]) return PS_ERR_INVALID_ARG;
+            if (!(lr_mult[q] == lr_mult[q]) || !(wd_mult[q] == wd_mult[q])) return PS_ERR_INVALID_ARG;
+        }
+        ps->num_layers = num_layers;
+        for (int q = 0; q < num_layers; ++q) {
+            ps->layer_end[q] = bounds[q + 1]; ps->layer_lr[q] = lr_mult[q]; ps->layer_wd[q] = wd_mult[q];
+        }
         return PS_OK;
     } PS_CATCH_ALL
 }
@@ -672,6 +886,7 @@ int ps_push_gradient_host(ps_t *ps, int learner, const void *grad_host, int64_t 
         DeviceGuard on_device(ps);
         const int rc = check_push(ps, learner, grad_host, ts);
         if (rc != PS_OK) return rc;
+        if (ps->n == 0) return push_common(ps, learner, nullptr, ts, -1);   // nothing to copy, nothing to stage
         if (!ps->staging) return PS_ERR_NO_STATE;
         if (ps->free_slots.empty()) return PS_ERR_QUEUE_FULL;
         const int slot = ps->free_slots.back();
@@ -716,7 +931,34 @@ int ps_push_slot(ps_t *ps, int learner, int slot_id, int64_t ts)
         const int rc = check_push(ps, learner, grad, ts);
         if (rc != PS_OK) return rc;                       // the learner keeps the slot and may try again
         ps->slot_lent[slot_id] = 0;
-        return push_common(ps, learner, grad, ts, slot_id);
+        return push_common(ps, learner, grad, ts, slot_id, true);
+    } PS_CATCH_ALL
+}
+
+int ps_slot_wait(ps_t *ps, int slot_id, void *stream)
+{
+    try {
+        if (!is_live(ps) || slot_id < 0 || slot_id >= ps->num_slots || !ps->slot_lent[slot_id]) return PS_ERR_INVALID_ARG;
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        if (st == ps->stream || !ps->slot_has_consumer[slot_id]) return PS_OK;   // stream order covers it / never read yet
+        DeviceGuard on_device(ps);
+        PS_CUDA(ps, cudaStreamWaitEvent(st, ps->slot_consumed[slot_id], 0));
+        return PS_OK;
+    } PS_CATCH_ALL
+}
+
+int ps_slot_written(ps_t *ps, int slot_id, void *stream)
+{
+    try {
+        if (!is_live(ps) || slot_id < 0 || slot_id >= ps->num_slots || !ps->slot_lent[slot_id]) return PS_ERR_INVALID_ARG;
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        if (st == ps->stream) return PS_OK;
+        DeviceGuard on_device(ps);
+        if (!ps->slot_filled[slot_id])
+            PS_CUDA(ps, cudaEventCreateWithFlags(&ps->slot_filled[slot_id], cudaEventDisableTiming));
+        PS_CUDA(ps, cudaEventRecord(ps->slot_filled[slot_id], st));
+        PS_CUDA(ps, cudaStreamWaitEvent(ps->stream, ps->slot_filled[slot_id], 0));
+        return PS_OK;
     } PS_CATCH_ALL
 }
 
@@ -727,6 +969,22 @@ int ps_synchronize(ps_t *ps)
         DeviceGuard on_device(ps);
         PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
         if (ps->copy_stream) PS_CUDA(ps, cudaStreamSynchronize(ps->copy_stream));
+        if (ps->bulk_status && ps->bulk_status->code != 0) return PS_ERR_DEVICE_WAIT;
+        return PS_OK;
+    } PS_CATCH_ALL
+}
+
+int ps_kernel_status(ps_t *ps, int *code, int *block, int64_t *tile, int *stage)
+{
+    try {
+        if (!is_live(ps)) return PS_ERR_INVALID_ARG;
+        DeviceGuard on_device(ps);
+        if (ps->device >= 0) PS_CUDA(ps, cudaStreamSynchronize(ps->stream));
+        const BulkStatus st = ps->bulk_status ? *ps->bulk_status : BulkStatus{0, 0, 0, 0};
+        if (code) *code = st.code;
+        if (block) *block = st.block;
+        if (tile) *tile = st.tile;
+        if (stage) *stage = st.stage;
         return PS_OK;
     } PS_CATCH_ALL
 }
@@ -842,6 +1100,7 @@ const char *ps_status_string(int status)
     case PS_ERR_NO_STATE: return "weights, momentum or staging slots not bound";
     case PS_ERR_LOG_EVICTED: return "log range not held";
     case PS_ERR_BARRIER: return "hardsync: learner already contributed to this round";
+    case PS_ERR_DEVICE_WAIT: return "an update kernel gave up on a bounded wait; re-initialise the weights";
     default: return status > 1 ? "updates applied" : "unknown status";
     }
 }

@@ -14,12 +14,22 @@ from typing import Callable, List, Optional
 import torch
 import torch.distributed as dist
 
-SHARD_ALIGN = 4          # elements: keeps every shard's base 16-byte aligned for the vector kernel
+SHARD_ALIGN = 4          # elements: 16 bytes of fp32, so theta, v and fp32 gradients keep the vector kernel
 
 
-def shard_bounds(num_params: int, world: int, align: int = SHARD_ALIGN) -> List[int]:
+def shard_align(grad_dtype: str = "fp32", bf16_arrays: bool = False) -> int:
+    """Elements a shard start must be a multiple of so that every array the server touches starts on a
+    16-byte boundary there: 4 for fp32 data, 8 as soon as bf16 gradients or a bf16 weight mirror are in
+    play (the vector kernel itself needs only 8 bytes for those, the bulk-copy kernel and copies 16)."""
+    return 8 if (grad_dtype == "bf16" or bf16_arrays) else SHARD_ALIGN
+
+
+def shard_bounds(num_params: int, world: int, align: int = 0, grad_dtype: str = "fp32",
+                 bf16_arrays: bool = False) -> List[int]:
     """world+1 offsets splitting [0, num_params) into contiguous ranges whose starts are multiples of
-    `align`; sizes differ by at most `align` and the last range takes the ragged end."""
+    `align` (default: shard_align of the data types); sizes differ by at most `align` and the last range
+    takes the ragged end."""
+    align = align or shard_align(grad_dtype, bf16_arrays)
     units = (num_params + align - 1) // align
     bounds = [min(num_params, (units * r // world) * align) for r in range(world)]
     return bounds + [num_params]
@@ -34,7 +44,7 @@ class ShardedParameterServer:
         self.world = dist.get_world_size(group) if dist.is_initialized() else 1
         self.rank = dist.get_rank(group) if dist.is_initialized() else 0
         self.num_params = int(num_params)
-        self.bounds = shard_bounds(self.num_params, self.world)
+        self.bounds = shard_bounds(self.num_params, self.world, grad_dtype=grad_dtype)
         self.lo, self.hi = self.bounds[self.rank], self.bounds[self.rank + 1]
         self.device = device
         if server_factory is None:
@@ -75,8 +85,21 @@ class ShardedParameterServer:
         return self.local.push_gradient(learner, grad_full[self.lo:self.hi], ts)
 
     def push_gradient_slice(self, learner: int, grad_slice: torch.Tensor, ts: int) -> bool:
-        assert grad_slice.numel() == self.hi - self.lo
+        """The scattered push: a learner sends every shard only that shard's range of its gradient
+        (elements [lo, hi) of this rank); nothing else of the gradient needs to exist on this rank."""
+        if grad_slice.numel() != self.hi - self.lo:
+            raise ValueError("slice of %d elements for a shard of %d" % (grad_slice.numel(), self.hi - self.lo))
         return self.local.push_gradient(learner, grad_slice, ts)
+
+    # receive slots of this rank's shard: a learner on the same GPU writes its slice straight into server memory
+    def bind_staging(self, num_slots: int) -> None:
+        self.local.bind_staging(num_slots)
+
+    def acquire_slot(self):
+        return self.local.acquire_slot()
+
+    def push_slot(self, learner: int, slot_id: int, ts: int) -> bool:
+        return self.local.push_slot(learner, slot_id, ts)
 
     def apply_update(self) -> int:
         return self.local.apply_update()

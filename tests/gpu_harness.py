@@ -39,8 +39,10 @@ def replay_gpu(ps: P.ParameterServer, kinds, learners, grad_fn, lazy: bool = Fal
 
 def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, grad_std, kinds, learners,
              w0: torch.Tensor, seed: int, fuse_t: int = 1, lazy: bool = False, precisions=(32, 64),
-             options=None, misalign: int = 0, checkpoints: int = 0, tol: float = 1e-5):
-    """Returns (gpu_w, gpu_v, gpu_log, {precision: (w, v, log)})."""
+             options=None, misalign: int = 0, checkpoints: int = 0, tol: float = 1e-5,
+             penalty_base=None, layers=None, mirror: bool = False):
+    """Returns (gpu_w, gpu_v, gpu_log, {precision: (w, v, log)}).  layers = (bounds, lr_mult, wd_mult);
+    mirror: also keep the bf16 weight mirror and compare it with the reference's rounding at the end."""
     dev = torch.device("cuda", 0)
     tdt = TORCH_DTYPE[grad_dtype]
     mod = P.binding.MODULATIONS[modulation]
@@ -48,6 +50,10 @@ def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, g
     for prec in precisions:
         r = R.ReferencePS(num_params, lam, n, alpha0, momentum, wd, mod, prec)
         r.set_weights(w0.numpy())
+        if penalty_base is not None:
+            r.set_penalty_base(penalty_base)
+        if layers is not None:
+            r.set_layer_multipliers(*layers)
         refs[prec] = r
 
     state = None
@@ -59,7 +65,12 @@ def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, g
                            device=dev, state=state)
     for key, val in (options or {}).items():
         ps.set_option(key, val)
+    if penalty_base is not None:
+        ps.set_penalty_base(penalty_base)
+    if layers is not None:
+        ps.set_layer_multipliers(*layers)
     ps.init_weights(w0.to(dev))
+    mirror_t = ps.bind_weight_mirror() if mirror else None
 
     def grad_fn(l, p):
         if misalign:
@@ -109,6 +120,13 @@ def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, g
     w = ps.w[:num_params].cpu().numpy().copy() if num_params else empty
     v = ps.v[:num_params].cpu().numpy().copy() if num_params else empty
     log = ps.update_log()
+    if mirror and 32 in refs and num_params:
+        got = mirror_t[:num_params].cpu().view(torch.int16).numpy().view(np.uint16)
+        assert np.array_equal(got, refs[32].weights_bf16()), "bf16 mirror differs from the reference's rounding"
+    run_pair.last_kernel = ps.get_option(P.PS_OPT_LAST_KERNEL)
+    run_pair.launches = {k: ps.get_option(o) for k, o in (("scalar", P.PS_OPT_LAUNCHES_SCALAR),
+                                                          ("vector", P.PS_OPT_LAUNCHES_VECTOR),
+                                                          ("bulk", P.PS_OPT_LAUNCHES_BULK))}
     ps.destroy()
     return w, v, log, out
 

@@ -32,7 +32,7 @@ def declared_symbols():
 
 def test_library_exports_every_declared_symbol():
     names = declared_symbols()
-    assert len(names) >= 18 and "ps_apply_update" in names
+    assert len(names) >= 30 and "ps_apply_update" in names and "ps_slot_wait" in names
     for n in names:
         assert hasattr(P.lib, n), n
     assert sorted(names) == sorted(P.binding.EXPORTS)
@@ -101,6 +101,112 @@ def test_schedule_matches_reference_bit_exactly(model, lam, n, mod, fuse_t, lazy
     assert P.ps_destroy(h) == 0
 
 
+@pytest.mark.parametrize("rho", [0.5, 0.75, 1.0])
+@pytest.mark.parametrize("fuse_t,lazy", [(1, False), (4, True)])
+def test_exponential_penalty_schedule_matches_reference(rho, fuse_t, lazy):
+    """Scales alpha0 * rho^tau / c, the decay coefficient and the logged staleness, bit for bit."""
+    lam, n, pushes = 12, 3, 480
+    kinds, learners = R.simulate_arrivals("exp", lam, pushes, 7)
+    ref = R.ReferencePS(0, lam, n, 0.02, 0.9, 5e-4, R.MOD_EXP_STALENESS, 32)
+    ref.set_penalty_base(rho)
+    nothing = np.zeros(0, np.float32)
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        ref.pull(l) if k == PULL else ref.push(l, nothing)
+    rlog = ref.log()
+    rc, h = make(lam, n, alpha0=0.02, mod=P.PS_MOD_EXP_STALENESS)
+    assert rc == 0 and P.ps_set_penalty_base(h, rho) == 0
+    drive(h, kinds, learners, fuse_t, lazy)
+    ts, log = fetch_log(h, lam // n)
+    assert ts == ref.timestamp
+    for f in ("update", "push_index", "ts_grad", "tau", "sigma", "learner", "position"):
+        assert np.array_equal(log[f], rlog[f]), f
+    assert np.array_equal(log["scale"], rlog["scale"].astype(np.float32))
+    assert np.array_equal(log["decay"], rlog["decay"].astype(np.float32))
+    assert np.array_equal(log["sigma"], log["tau"]) and log["tau"].max() > 4
+    P.ps_destroy(h)
+
+
+def test_penalty_base_and_layer_table_argument_checks():
+    rc, h = make(2, 1, num_params=0)
+    for bad in (0.0, -0.5, 1.5, float("nan")):
+        assert P.ps_set_penalty_base(h, bad) == P.PS_ERR_INVALID_ARG
+    assert P.ps_set_penalty_base(h, 1.0) == 0
+    b0 = np.array([0, 0, 0], np.int64)
+    one = np.ones(2, np.float32)
+    assert P.ps_set_layer_multipliers(h, 2, b0.ctypes.data, one.ctypes.data, one.ctypes.data) == 0   # empty layers are fine
+    assert P.ps_set_layer_multipliers(h, 0, None, None, None) == 0
+    assert P.ps_set_layer_multipliers(h, 2, None, one.ctypes.data, one.ctypes.data) == P.PS_ERR_INVALID_ARG
+    assert P.ps_set_layer_multipliers(h, P.PS_MAX_LAYERS + 1, b0.ctypes.data, one.ctypes.data, one.ctypes.data) == P.PS_ERR_INVALID_ARG
+    bad = np.array([0, 1, 0], np.int64)                                         # does not end at num_params
+    assert P.ps_set_layer_multipliers(h, 2, bad.ctypes.data, one.ctypes.data, one.ctypes.data) == P.PS_ERR_INVALID_ARG
+    nan = np.array([1.0, np.nan], np.float32)
+    assert P.ps_set_layer_multipliers(h, 2, b0.ctypes.data, nan.ctypes.data, one.ctypes.data) == P.PS_ERR_INVALID_ARG
+    assert P.ps_push_gradient(h, 0, FAKE_GRAD, 0) == P.PS_OK                    # a gradient is pending now
+    assert P.ps_set_penalty_base(h, 0.5) == P.PS_ERR_INVALID_ARG
+    assert P.ps_set_layer_multipliers(h, 2, b0.ctypes.data, one.ctypes.data, one.ctypes.data) == P.PS_ERR_INVALID_ARG
+    P.ps_destroy(h)
+    h2 = C.c_void_p()
+    assert P.ps_create(C.byref(h2), 0, 2, 1, 0.1, 0.0, 0.0, 3) == P.PS_ERR_INVALID_ARG     # no such modulation
+
+
+def test_read_only_options_and_kernel_options():
+    rc, h = make(7, 2)
+    v = C.c_int64()
+    assert P.ps_get_option(h, P.PS_OPT_GROUP_SIZE, C.byref(v)) == 0 and v.value == 3        # floor(7 / 2)
+    for key in (P.PS_OPT_LAST_KERNEL, P.PS_OPT_LAUNCHES_SCALAR, P.PS_OPT_LAUNCHES_VECTOR, P.PS_OPT_LAUNCHES_BULK):
+        assert P.ps_get_option(h, key, C.byref(v)) == 0 and v.value == 0
+        assert P.ps_set_option(h, key, 1) == P.PS_ERR_INVALID_ARG
+    assert P.ps_set_option(h, P.PS_OPT_GROUP_SIZE, 4) == P.PS_ERR_INVALID_ARG
+    assert P.ps_set_option(h, P.PS_OPT_KERNEL, P.PS_KERNEL_BULK) == 0
+    assert P.ps_set_option(h, P.PS_OPT_KERNEL, 4) == P.PS_ERR_INVALID_ARG
+    for key, good, bads in ((P.PS_OPT_BULK_TILE, (0, 256, 1024, 8192), (100, 384, 16384, -1)),
+                            (P.PS_OPT_BULK_STAGES, (2, 8), (1, 9)),
+                            (P.PS_OPT_BULK_WAIT_LIMIT, (16, 1 << 20), (0, 15)),
+                            (P.PS_OPT_BULK_SELFTEST, (0, 1), (2, -1))):
+        for g in good:
+            assert P.ps_set_option(h, key, g) == 0
+            assert P.ps_get_option(h, key, C.byref(v)) == 0 and v.value == g
+        for b in bads:
+            assert P.ps_set_option(h, key, b) == P.PS_ERR_INVALID_ARG
+    code, tile = C.c_int(-1), C.c_int64(-1)
+    assert P.ps_kernel_status(h, C.byref(code), None, C.byref(tile), None) == 0 and code.value == 0
+    P.ps_destroy(h)
+
+
+def test_binding_refuses_tensors_the_kernel_would_misread():
+    """The library sees addresses only; the binding checks type, length, layout and placement before it
+    hands one over.  Nothing here launches a kernel."""
+    import torch
+    from paper_1511_05950_b200.binding import require_tensor
+    f32, bf = torch.float32, torch.bfloat16
+    require_tensor(torch.zeros(16), f32, 16, "x", on_gpu=False)
+    require_tensor(torch.zeros(20)[2:18], f32, 16, "x", on_gpu=False)       # an offset view is fine
+    with pytest.raises(TypeError):
+        require_tensor(torch.zeros(16, dtype=bf), f32, 16, "x", on_gpu=False)          # would read 4N bytes of a 2N buffer
+    with pytest.raises(TypeError):
+        require_tensor(torch.zeros(16, dtype=torch.float64), f32, 16, "x", on_gpu=False)
+    with pytest.raises(ValueError):
+        require_tensor(torch.zeros(15), f32, 16, "x", on_gpu=False)                   # too short
+    with pytest.raises(ValueError):
+        require_tensor(torch.zeros(32)[::2], f32, 16, "x", on_gpu=False)              # strided
+    with pytest.raises(ValueError):
+        require_tensor(torch.zeros(16), f32, 16, "x", on_gpu=True)                    # host memory as a device operand
+    # through the class, on a server without parameters (no GPU needed): the element type is still checked
+    ps = P.ParameterServer(0, 2, 1, 0.1)
+    with pytest.raises(TypeError):
+        ps.push_gradient(0, torch.zeros(0, dtype=bf), 0)
+    with pytest.raises(TypeError):
+        ps.pull_weights(torch.zeros(0, dtype=torch.float16))
+    with pytest.raises(TypeError):
+        ps.init_weights(torch.zeros(0, dtype=torch.float64))
+    assert ps.timestamps() == (0, 0)                                        # nothing reached the server
+    ps.destroy()
+    b16 = P.ParameterServer(0, 2, 1, 0.1, grad_dtype="bf16")
+    with pytest.raises(TypeError):
+        b16.push_gradient(0, torch.zeros(0), 0)                             # fp32 into a bf16 server
+    b16.destroy()
+
+
 def test_rate_schedule_applies_to_later_pushes_only():
     rc, h = make(2, 1, alpha0=0.5, m=0.0, wd=0.0)
     assert P.ps_push_gradient(h, 0, FAKE_GRAD, 0) == P.PS_OK
@@ -147,7 +253,6 @@ def test_error_codes():
     assert P.ps_push_gradient(h, 0, FAKE_GRAD, 1) == P.PS_ERR_BAD_TIMESTAMP       # from the future: tau < 0
     assert P.ps_push_gradient(h, 0, FAKE_GRAD, -1) == P.PS_ERR_BAD_TIMESTAMP
     assert P.ps_push_gradient(h, 0, FAKE_GRAD + 2, 0) == P.PS_ERR_INVALID_ARG     # fp32 needs 4-byte alignment
-    assert P.ps_push_gradient_host(h, 0, FAKE_GRAD, 0) == P.PS_ERR_NO_STATE       # no staging slots bound
     assert P.ps_apply_update(h) == P.PS_ERR_NOT_READY
     assert P.ps_push_gradient(h, 0, FAKE_GRAD, 0) == P.PS_OK
     assert P.ps_push_gradient(h, 1, FAKE_GRAD, 0) == P.PS_OK

@@ -52,3 +52,19 @@ def test_steps_group_trace_events_by_completed_update():
     for evs in steps:
         assert sum(k == 1 for k, _ in evs) == cfg.c and evs[-1][0] == 1
     assert bench.algorithmic_bytes(60965224, 4, 4) == 60965224 * 32
+
+
+def test_traffic_is_reported_only_for_the_captured_kernel_instantiation():
+    v, src = bench.traffic_for("large_softsync", "vector", "fp32", 4, 1, 0, False, False)
+    assert v == 1.913e9 and os.path.exists(os.path.join(os.path.dirname(bench.__file__), src))
+    for other in (("large_softsync", "bulk", "fp32", 4, 1, 0, False, False),        # another kernel
+                  ("large_softsync", "vector", "fp32", 4, 1, 256, False, False),    # another block size
+                  ("large_softsync", "vector", "fp32", 4, 1, 0, True, False),       # with the bf16 mirror
+                  ("large_softsync@flat16777216", "vector", "fp32", 4, 1, 0, False, False)):
+        v, why = bench.traffic_for(*other)
+        assert v is None and "no ncu capture" in why
+
+
+def test_repeats_are_summarised_by_their_median():
+    stat = bench.summarise([{"ms": 30.0}, {"ms": 10.0}, {"ms": 20.0}], 10)
+    assert stat == {"median": 2.0, "min": 1.0, "max": 3.0}

@@ -7,7 +7,12 @@ timestamp it pulled.  Images are class templates plus noise (CIFAR10 itself is n
 reports, and this checks: alpha0 is a good rate for one learner; with 30 asynchronous learners the same constant
 alpha0 does not train at all, and dividing it by the staleness trains to high accuracy.
 The learners use PyTorch; everything the server does runs in the library under test.
+
+Every gradient the learners push (real autograd gradients: a large dynamic range, exact zeros from dead
+units, values growing without bound in the run that diverges) is also pushed, with the same timestamp, into
+the CPU reference; the final weights, momentum and the whole log must equal the reference's bit for bit.
 """
+import numpy as np
 import pytest
 import torch
 import torch.nn.functional as F
@@ -32,6 +37,8 @@ def _forward(layout, flat, x):
 
 def _train(num_learners, n, modulation, pushes, mu=8):
     import paper_1511_05950_b200 as P
+    from oracle import reference as R
+    from tests.gpu_harness import assert_logs_equal
     from workloads import arrivals, generators as G, layouts
 
     dev = torch.device("cuda", 0)
@@ -53,7 +60,10 @@ def _train(num_learners, n, modulation, pushes, mu=8):
 
     kinds, learners = arrivals.make_trace("uniform", num_learners, pushes, 5)
     ps = P.ParameterServer(num_params, num_learners, n, ALPHA0, 0.9, 5e-4, modulation, device=dev)
-    ps.init_weights(G.initial_weights(layout, 3, 0.05, device=dev))
+    w0 = G.initial_weights(layout, 3, 0.05, device=dev)
+    ps.init_weights(w0)
+    ref = R.ReferencePS(num_params, num_learners, n, ALPHA0, 0.9, 5e-4, P.binding.MODULATIONS[modulation], 32)
+    ref.set_weights(w0.cpu().numpy())
     held = {l: torch.empty(num_params, device=dev) for l in range(num_learners)}
     stamp = {}
     g = torch.Generator(device=dev)
@@ -65,9 +75,18 @@ def _train(num_learners, n, modulation, pushes, mu=8):
             w_l = held[l].clone().requires_grad_(True)
             x, y = batch(mu, g)
             grad, = torch.autograd.grad(F.cross_entropy(_forward(layout, w_l, x), y), w_l)    # calcGradient
-            if ps.push_gradient(l, grad.contiguous(), stamp[l]):      # pushGradient
+            grad = grad.contiguous()
+            ref.push(l, grad.cpu().numpy(), timestamp=stamp[l])
+            if ps.push_gradient(l, grad, stamp[l]):                   # pushGradient
                 ps.apply_update()
     ps.synchronize()
+    w32, v32 = ref.state()
+    w_gpu, v_gpu = ps.w.cpu().numpy(), ps.v.cpu().numpy()
+    # exact equality of every value; a run that has diverged must have its inf / nan in the same places
+    # (the payload bits of a nan are the one thing CPU and GPU arithmetic may legitimately choose differently)
+    assert np.array_equal(w_gpu, w32.astype(np.float32), equal_nan=True)
+    assert np.array_equal(v_gpu, v32.astype(np.float32), equal_nan=True)
+    assert_logs_equal(ps.update_log(), ref.log())
     with torch.no_grad():
         accuracy = (_forward(layout, ps.w, xv).argmax(1) == yv).float().mean().item()
     tau = ps.update_log()["tau"]

@@ -115,6 +115,154 @@ def test_large_stale_bf16_full_size():
     assert len(log) == 2000 and log["tau"].max() > 100
 
 
+class PartitionedReference:
+    """The unmodified reference on the whole vector, one instance per contiguous range and host thread (the
+    update is element-wise, so the ranges are independent; the C calls release the interpreter lock)."""
+
+    def __init__(self, cfg, w0: np.ndarray, threads: int, layers=None):
+        from concurrent.futures import ThreadPoolExecutor
+        n = w0.size
+        self.bounds = [n * t // threads for t in range(threads + 1)]
+        self.pool = ThreadPoolExecutor(threads)
+        self.parts = []
+        for a, b in zip(self.bounds[:-1], self.bounds[1:]):
+            r = R.ReferencePS(b - a, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
+                              P.binding.MODULATIONS[cfg.modulation], 32)
+            r.set_weights(w0[a:b])
+            if layers is not None:                       # the layer table restricted to [a, b)
+                bounds, lm, dm = layers
+                cut = [min(max(x, a), b) - a for x in bounds]
+                r.set_layer_multipliers(cut, lm, dm)
+            self.parts.append((a, b, r))
+
+    def pull(self, learner):
+        return [r.pull(learner) for _, _, r in self.parts][0]
+
+    def push(self, learner, grad: np.ndarray):
+        list(self.pool.map(lambda part: part[2].push(learner, grad[part[0]:part[1]]), self.parts))
+
+    def assert_state_equals(self, w: np.ndarray, v: np.ndarray):
+        for a, b, r in self.parts:
+            wr, vr = r.state()
+            assert np.array_equal(w[a:b], wr.astype(np.float32)), "weights differ in [%d, %d)" % (a, b)
+            assert np.array_equal(v[a:b], vr.astype(np.float32)), "momentum differs in [%d, %d)" % (a, b)
+
+    def close(self):
+        self.pool.shutdown()
+        for _, _, r in self.parts:
+            r.close()
+
+
+@pytest.mark.parametrize("cfg,updates,layers", [
+    (configs.LARGE_SOFTSYNC, 16, False), (configs.LARGE_STALE_BF16, 32, False), (configs.LARGE_SOFTSYNC, 4, True)],
+    ids=["large_softsync", "large_stale_bf16", "large_softsync_layer_multipliers"])
+def test_every_element_at_full_size(cfg, updates, layers):
+    """Configs 3 and 4 on the whole 60,965,224-element vector in the launch mode bench.py times
+    (programmatic dependent launches, T = 8 for the bf16 case), an even number of launches so that both
+    traversal directions and overlapped pairs occur: EVERY element of theta and v bit-equal to the fp32
+    reference, the log equal.  Third case: the same with Caffe-style per-layer multipliers."""
+    import os
+    from tests.test_gpu_parity import caffe_style_multipliers
+    dev = torch.device("cuda", 0)
+    layout = cfg.layout()
+    n = layout.num_params
+    tdt = TORCH_DTYPE[cfg.grad_dtype]
+    pushes = updates * cfg.c
+    table = caffe_style_multipliers(layout) if layers else None
+    kinds, learners = R.simulate_arrivals(cfg.arrival_model, cfg.num_learners, pushes, cfg.seed)
+    w0 = G.initial_weights(layout, cfg.seed, cfg.weight_std, device=dev)
+    ref = PartitionedReference(cfg, w0.cpu().numpy(), max(1, min(32, os.cpu_count() or 1)), table)
+    ps = P.ParameterServer(n, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
+                           cfg.modulation, cfg.grad_dtype, cfg.fuse_t, device=dev)
+    if table:
+        ps.set_layer_multipliers(*table)
+    ps.init_weights(w0)
+    ps.set_option(P.PS_OPT_OVERLAP_LAUNCH, 1)
+    pulled, counts, ready, held = {}, {}, 0, []
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == PULL:
+            pulled[l] = ps.pull_weights()
+            assert ref.pull(l) == pulled[l]
+            continue
+        p = counts.get(l, 0)
+        counts[l] = p + 1
+        g = G.gradient(cfg.seed, l, p, n, cfg.grad_std, dtype=tdt, device=dev)
+        ref.push(l, as_reference_grad(g))                  # the device-to-host copy also completes the gradient
+        ready += ps.push_gradient(l, g, pulled[l])
+        if ready >= cfg.fuse_t:
+            ready -= ps.apply_update()                     # back-to-back launches overlap when the next group is ready
+    ps.flush(); ps.synchronize()
+    launches = ps.get_option(P.PS_OPT_LAUNCHES_VECTOR)
+    assert launches == updates // cfg.fuse_t and launches % 2 == 0 and ps.get_option(P.PS_OPT_LAUNCHES_SCALAR) == 0
+    ref.assert_state_equals(ps.w.cpu().numpy(), ps.v.cpu().numpy())
+    assert_logs_equal(ps.update_log(), ref.parts[0][2].log())
+    ps.destroy()
+    ref.close()
+
+
+@pytest.mark.parametrize("align", [4, 0], ids=["starts_8_byte_aligned", "starts_16_byte_aligned"])
+def test_eight_shards_of_the_bf16_config_keep_the_vector_kernel(align):
+    """Config 4 (bf16 gradients, T = 8) cut into the eight contiguous shards an 8-GPU server would use, all
+    on this GPU: every shard's pointers satisfy the vector kernel (bf16 gradient slices are only 8-byte
+    aligned at some shard starts), every launch reports the vector kernel, and the shards together equal
+    the unsharded server on every element and the reference on sampled ones."""
+    from paper_1511_05950_b200.sharded import shard_bounds
+    cfg = configs.LARGE_STALE_BF16
+    dev = torch.device("cuda", 0)
+    layout = cfg.layout()
+    n = layout.num_params
+    bounds = shard_bounds(n, 8, align=align, grad_dtype="bf16")
+    if align == 4:                                          # the split an fp32 server would use
+        assert any((2 * b) % 16 == 8 for b in bounds[1:-1])
+    else:                                                   # the split the sharded server picks for bf16 gradients
+        assert all((2 * b) % 16 == 0 for b in bounds[1:-1])
+    pushes = 16
+    idx = sample_indices(layout, 4000, 2)
+    idx_dev = idx.to(dev)
+    kinds, learners = R.simulate_arrivals(cfg.arrival_model, cfg.num_learners, pushes, cfg.seed)
+    ref = R.ReferencePS(idx.numel(), cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
+                        P.binding.MODULATIONS[cfg.modulation], 32)
+    ref.set_weights(G.initial_weights_at(layout, cfg.seed, idx, cfg.weight_std).numpy())
+    w0 = G.initial_weights(layout, cfg.seed, cfg.weight_std, device=dev)
+    whole = P.ParameterServer(n, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
+                              cfg.modulation, "bf16", 8, device=dev)
+    whole.init_weights(w0)
+    wbuf, vbuf = torch.empty(n, device=dev), torch.empty(n, device=dev)
+    shards = []
+    for a, b in zip(bounds[:-1], bounds[1:]):
+        sh = P.ParameterServer(b - a, cfg.num_learners, cfg.n, cfg.alpha0, cfg.momentum, cfg.weight_decay,
+                               cfg.modulation, "bf16", 8, device=dev, state=(wbuf[a:b], vbuf[a:b]))
+        sh.set_option(P.PS_OPT_KERNEL, P.PS_KERNEL_VECTOR)          # a scalar fallback would be an error
+        sh.init_weights(w0[a:b])
+        shards.append((a, b, sh))
+    pulled, counts = {}, {}
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == PULL:
+            pulled[l] = whole.pull_weights()
+            assert ref.pull(l) == pulled[l]
+            assert all(sh.pull_weights() == pulled[l] for _, _, sh in shards)
+            continue
+        p = counts.get(l, 0); counts[l] = p + 1
+        g = G.gradient(cfg.seed, l, p, n, cfg.grad_std, dtype=torch.bfloat16, device=dev)
+        ref.push(l, as_reference_grad(G.gradient_at(cfg.seed, l, p, idx, cfg.grad_std, dtype=torch.bfloat16)))
+        whole.push_gradient(l, g, pulled[l])
+        for a, b, sh in shards:
+            sh.push_gradient(l, g[a:b], pulled[l])
+    assert whole.flush() == 16
+    for a, b, sh in shards:
+        assert sh.flush() == 16
+        assert sh.get_option(P.PS_OPT_LAST_KERNEL) == P.PS_KERNEL_VECTOR
+        assert sh.get_option(P.PS_OPT_LAUNCHES_VECTOR) == 2 and sh.get_option(P.PS_OPT_LAUNCHES_SCALAR) == 0
+    torch.cuda.synchronize()
+    assert torch.equal(whole.w, wbuf) and torch.equal(whole.v, vbuf)
+    w32, v32 = ref.state()
+    assert np.array_equal(wbuf[idx_dev].cpu().numpy(), w32.astype(np.float32))
+    assert np.array_equal(vbuf[idx_dev].cpu().numpy(), v32.astype(np.float32))
+    for _, _, sh in shards:
+        sh.destroy()
+    whole.destroy()
+
+
 @pytest.mark.parametrize("grad_dtype", ["fp32", "bf16"])
 def test_more_than_two_to_the_thirty_elements(grad_dtype):
     """A ragged vector of 2^30 + 3 elements (the sweep's largest size): byte offsets beyond 2^32, the

@@ -62,6 +62,7 @@ def test_large_stale_bf16_scaled_down(lazy):
 
 
 def _simple(num_params, lam, n, pushes, grad_dtype="fp32", model="exp", seed=77, **kw):
+    """Random arrivals on a flat vector with the usual hyper-parameters, compared with both references."""
     kinds, learners = R.simulate_arrivals(model, lam, pushes, seed)
     w0 = G.initial_weights(layouts.flat(num_params), seed) if num_params else torch.zeros(0)
     w, v, log, refs = run_pair(num_params, lam, n, 0.01, 0.9, 5e-4, "inv_staleness", grad_dtype, 1e-3,
@@ -105,10 +106,161 @@ def test_temporal_fusion_is_invisible(lam, n, fuse_t, grad_dtype):
     {P.PS_OPT_KERNEL: P.PS_KERNEL_SCALAR}, {P.PS_OPT_KERNEL: P.PS_KERNEL_VECTOR},
     {P.PS_OPT_BLOCK_THREADS: 128}, {P.PS_OPT_BLOCK_THREADS: 256}, {P.PS_OPT_BLOCK_THREADS: 512},
     {P.PS_OPT_KERNEL: P.PS_KERNEL_SCALAR, P.PS_OPT_BLOCK_THREADS: 512},
+    {P.PS_OPT_KERNEL: P.PS_KERNEL_BULK},
+    {P.PS_OPT_KERNEL: P.PS_KERNEL_BULK, P.PS_OPT_BULK_TILE: 256, P.PS_OPT_BULK_STAGES: 2},
+    {P.PS_OPT_KERNEL: P.PS_KERNEL_BULK, P.PS_OPT_BULK_TILE: 512, P.PS_OPT_BULK_STAGES: 8, P.PS_OPT_BLOCK_THREADS: 128},
+    {P.PS_OPT_KERNEL: P.PS_KERNEL_BULK, P.PS_OPT_BULK_TILE: 1024, P.PS_OPT_BULK_STAGES: 3, P.PS_OPT_OVERLAP_LAUNCH: 1},
 ])
 def test_launch_shape_does_not_change_the_bits(options):
-    _simple(70001, 8, 2, 40, "fp32", options=options)
-    _simple(70001, 8, 2, 40, "bf16", options=options)
+    want = {P.PS_KERNEL_SCALAR: "scalar", P.PS_KERNEL_BULK: "bulk"}.get(options.get(P.PS_OPT_KERNEL), "vector")
+    for grad_dtype in ("fp32", "bf16"):
+        _simple(70001, 8, 2, 40, grad_dtype, options=options)
+        launches = run_pair.launches
+        assert launches[want] == 10 and sum(launches.values()) == 10        # the kernel asked for is the one that ran
+        assert run_pair.last_kernel == P.binding.KERNELS[want]
+
+
+@pytest.mark.parametrize("grad_dtype,fuse_t,lam,n", [("fp32", 1, 8, 2), ("bf16", 8, 6, 6), ("fp32", 4, 8, 2), ("bf16", 1, 16, 1)])
+def test_bulk_copy_kernel_matches_reference(grad_dtype, fuse_t, lam, n):
+    """The shared-memory staged kernel on a vector of many tiles and a ragged end, both traversal directions
+    (launches alternate), with temporal fusion, the bf16 mirror and a layer table whose boundaries cut
+    fragments and tiles."""
+    n_el = 37 * 4096 + 1234 + 3
+    bounds = [0, 4096, 4097, 4097, 10001, 3 * 4096 + 2, 20 * 4096, n_el - 5, n_el]
+    layers = (bounds, [1.0, 2.0, 3.0, 0.5, 1.0, 2.0, 0.25, 1.5], [1.0, 0.0, 1.0, 2.0, 1.0, 0.0, 1.0, 3.0])
+    for use_layers in (None, layers):
+        _simple(n_el, lam, n, 12 * (lam // n) * fuse_t, grad_dtype, model="lognormal", fuse_t=fuse_t, lazy=fuse_t > 1,
+                options={P.PS_OPT_KERNEL: P.PS_KERNEL_BULK, P.PS_OPT_BULK_TILE: 2048 if fuse_t < 8 else 0},
+                layers=use_layers, mirror=True)
+        assert run_pair.launches["bulk"] == 12 and run_pair.launches["vector"] == 0
+
+
+def test_bulk_copy_kernel_refuses_what_it_cannot_stage():
+    """More than 16 gradients per launch, or a pointer that is not 16-byte aligned: an error, not a fallback."""
+    dev = torch.device("cuda", 0)
+    ps = P.ParameterServer(8192, 17, 1, 0.01, device=dev)
+    ps.set_option(P.PS_OPT_KERNEL, P.PS_KERNEL_BULK)
+    ps.init_weights(torch.zeros(8192))
+    g = torch.zeros(8192, device=dev)
+    for l in range(17):
+        ps.push_gradient(l, g, 0)
+    with pytest.raises(P.SoftsyncError) as e:
+        ps.apply_update()
+    assert e.value.status == P.PS_ERR_INVALID_ARG and ps.timestamps() == (0, 1)
+    ps.set_option(P.PS_OPT_KERNEL, P.PS_KERNEL_AUTO)
+    assert ps.apply_update() == 1
+    ps.destroy()
+    ps = P.ParameterServer(8192, 1, 1, 0.01, grad_dtype="bf16", device=dev)
+    ps.set_option(P.PS_OPT_KERNEL, P.PS_KERNEL_BULK)
+    ps.init_weights(torch.zeros(8192))
+    buf = torch.zeros(8192 + 8, dtype=torch.bfloat16, device=dev)
+    ps.push_gradient(0, buf[4:4 + 8192], 0)                 # 8-byte aligned: fine for the vector kernel only
+    with pytest.raises(P.SoftsyncError):
+        ps.apply_update()
+    ps.set_option(P.PS_OPT_KERNEL, P.PS_KERNEL_VECTOR)
+    assert ps.apply_update() == 1 and ps.get_option(P.PS_OPT_LAST_KERNEL) == P.PS_KERNEL_VECTOR
+    ps.destroy()
+
+
+def test_bulk_copy_kernel_wait_runs_out_and_is_reported():
+    """A copy barrier that never completes (one block is told to expect 16 bytes that nothing sends): the
+    block's bounded wait runs out, the kernel returns by itself, the host reads the status record, and
+    the context stays usable: after re-initialising, the same server matches the reference."""
+    from tests.gpu_harness import as_reference_grad
+    dev = torch.device("cuda", 0)
+    n_el, lam = 64 * 1024 + 7, 2
+    w0 = G.initial_weights(layouts.flat(n_el), 51)
+    ps = P.ParameterServer(n_el, lam, 1, 0.01, 0.9, 5e-4, device=dev)
+    ps.set_option(P.PS_OPT_KERNEL, P.PS_KERNEL_BULK)
+    ps.set_option(P.PS_OPT_BULK_TILE, 1024)
+    ps.set_option(P.PS_OPT_BULK_WAIT_LIMIT, 2000)
+    ps.init_weights(w0.to(dev))
+    grads = [G.gradient(51, l, 0, n_el, 1e-3, device=dev) for l in range(lam)]
+    ps.set_option(P.PS_OPT_BULK_SELFTEST, 1)
+    for l in range(lam):
+        ps.push_gradient(l, grads[l], 0)
+    assert ps.apply_update() == 1                          # the launch itself is fine
+    with pytest.raises(P.SoftsyncError) as e:
+        ps.synchronize()
+    assert e.value.status == P.PS_ERR_DEVICE_WAIT
+    code, block, tile, stage = ps.kernel_status()
+    assert (code, block, tile, stage) == (1, 0, 0, 0)
+    assert ps.get_option(P.PS_OPT_BULK_SELFTEST) == 0      # one launch only
+    torch.cuda.synchronize()                               # the context is intact
+    ps.init_weights(w0.to(dev))                            # theta and v were partly updated: start again
+    ps.synchronize()
+    assert ps.kernel_status()[0] == 0
+    ref = R.ReferencePS(n_el, lam, 1, 0.01, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    for u in range(3):
+        ts = ps.pull_weights()
+        for l in range(lam):
+            ref.pull(l)
+        for l in range(lam):
+            g = G.gradient(51, l, u, n_el, 1e-3, device=dev)
+            ref.push(l, as_reference_grad(g))
+            ps.push_gradient(l, g, ts)
+        assert ps.apply_update() == 1
+    ps.synchronize()
+    assert np.array_equal(ps.w.cpu().numpy(), ref.state()[0].astype(np.float32))
+    assert np.array_equal(ps.v.cpu().numpy(), ref.state()[1].astype(np.float32))
+    ps.destroy()
+
+
+@pytest.mark.parametrize("rho", [0.5, 0.9])
+@pytest.mark.parametrize("grad_dtype,fuse_t", [("fp32", 1), ("bf16", 4)])
+def test_exponential_penalty_matches_reference(rho, grad_dtype, fuse_t):
+    """alpha = alpha0 * rho^tau (the rule Section 1 contrasts with Eq. 3) on an Exp(1) arrival trace with
+    staleness up to several tens."""
+    kinds, learners = R.simulate_arrivals("exp", 12, 240, 61)
+    n_el = 50001
+    w0 = G.initial_weights(layouts.flat(n_el), 61)
+    w, v, log, refs = run_pair(n_el, 12, 6, 0.02, 0.9, 5e-4, "exp_staleness", grad_dtype, 1e-3, kinds, learners, w0, 61,
+                               fuse_t=fuse_t, lazy=fuse_t > 1, penalty_base=rho)
+    assert_parity(w, v, log, refs, TOL_BF16 if grad_dtype == "bf16" else TOL_FP32)
+    assert log["tau"].max() >= 5 and np.array_equal(log["sigma"], log["tau"])
+    assert len(np.unique(log["scale"])) >= 5
+
+
+def caffe_style_multipliers(layout):
+    """Rate x1 / decay x1 for weights, rate x2 / decay x0 for biases (the usual setting of the Caffe models
+    that Section 4.1's networks follow)."""
+    bounds = [seg.offset for seg in layout.segments] + [layout.num_params]
+    return (bounds, [2.0 if seg.is_bias else 1.0 for seg in layout.segments],
+            [0.0 if seg.is_bias else 1.0 for seg in layout.segments])
+
+
+@pytest.mark.parametrize("kernel", ["vector", "scalar", "bulk"])
+def test_layer_multipliers_on_the_small_network(kernel):
+    """Config 1 (89,578 elements, N mod 4 = 2, layer boundaries at every residue mod 4) with per-layer
+    multipliers, every element compared."""
+    cfg = configs.TINY_SOFTSYNC
+    layout = cfg.layout()
+    worst, log = run_config(cfg, num_pushes=160, layers=caffe_style_multipliers(layout),
+                            options={P.PS_OPT_KERNEL: P.binding.KERNELS[kernel], P.PS_OPT_BULK_TILE: 512})
+    assert run_pair.launches[kernel] == 40
+    worst, log = run_config(configs.PURE_ASYNC, num_pushes=300, layers=caffe_style_multipliers(layout), fuse_t=8, lazy=True,
+                            options={P.PS_OPT_KERNEL: P.binding.KERNELS[kernel]})
+
+
+@pytest.mark.parametrize("grad_dtype,fuse_t,lam,n", [("fp32", 1, 6, 2), ("bf16", 3, 4, 4), ("fp32", 16, 40, 2), ("bf16", 1, 20, 1)])
+def test_layer_boundaries_anywhere(grad_dtype, fuse_t, lam, n):
+    """Boundaries inside fragments, empty layers, a one-element layer, a frozen layer (rate x0), layers that
+    end in the ragged tail; all-ones multipliers give the bits of a server without a table."""
+    n_el = 20003
+    bounds = [0, 1, 1, 6, 7, 4098, 4099, 4099, 9001, 15002, 20000, 20002, n_el]
+    lm = [1.0, 3.0, 0.5, 2.0, 1.0, 0.0, 1.0, 2.0, 0.125, 1.0, 4.0, 1.5]
+    dm = [1.0, 1.0, 0.0, 2.0, 1.0, 1.0, 5.0, 0.0, 1.0, 0.5, 1.0, 0.0]
+    pushes = 10 * (lam // n) * min(fuse_t, 4)
+    a = _simple(n_el, lam, n, pushes, grad_dtype, model="lognormal", fuse_t=fuse_t, lazy=fuse_t > 1, layers=(bounds, lm, dm), mirror=True)
+    assert run_pair.launches["vector"] > 0 and run_pair.launches["scalar"] == 0
+    ones = _simple(n_el, lam, n, pushes, grad_dtype, model="lognormal", fuse_t=fuse_t, lazy=fuse_t > 1,
+                   layers=([0, 5, n_el], [1.0, 1.0], [1.0, 1.0]))
+    none = _simple(n_el, lam, n, pushes, grad_dtype, model="lognormal", fuse_t=fuse_t, lazy=fuse_t > 1)
+    assert np.array_equal(ones[0], none[0]) and np.array_equal(ones[1], none[1])
+    assert not np.array_equal(a[0], none[0])
+    w0 = G.initial_weights(layouts.flat(n_el), 77).numpy()
+    assert np.array_equal(a[0][4098:4099], w0[4098:4099])          # the frozen layer did not move
 
 
 @pytest.mark.parametrize("grad_dtype", ["fp32", "bf16"])
@@ -227,7 +379,53 @@ def test_overlapped_launch_gives_the_same_bits(grad_dtype, fuse_t):
     from tests.gpu_harness import as_reference_grad
     from tests.helpers import replay_reference
     replay_reference(ref, kinds, learners, lambda l, b: as_reference_grad(grads[(l, b)]))
-    assert np.array_equal(results[1][0], ref.state()[0].astype(np.float32))
+    from tests.gpu_harness import assert_logs_equal
+    for w, v, log in results:
+        assert np.array_equal(w, ref.state()[0].astype(np.float32)) and np.array_equal(v, ref.state()[1].astype(np.float32))
+        assert_logs_equal(log, ref.log())
+
+
+@pytest.mark.parametrize("grad_dtype,fuse_t", [("fp32", 1), ("bf16", 2)])
+def test_overlapped_launch_with_host_gradients_in_recycled_slots(grad_dtype, fuse_t):
+    """The arrangement the benchmark's end-to-end leg runs: programmatic dependent launches while every
+    gradient arrives from pinned host memory into 2*c*T staging slots that are reused generation after
+    generation, the copy of the next gradients enqueued right behind the kernel that still reads the
+    previous ones.  Against the reference, every element."""
+    from tests.gpu_harness import as_reference_grad, assert_logs_equal
+    dev = torch.device("cuda", 0)
+    n_el, lam, n = 2_000_003, 6, 2
+    c = lam // n
+    tdt = torch.bfloat16 if grad_dtype == "bf16" else torch.float32
+    pushes = 2 * c * fuse_t * 5                              # five generations of every slot
+    kinds, learners = R.simulate_arrivals("uniform", lam, pushes, 33)
+    w0 = G.initial_weights(layouts.flat(n_el), 33)
+    ref = R.ReferencePS(n_el, lam, n, 0.01, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    ps = P.ParameterServer(n_el, lam, n, 0.01, 0.9, 5e-4, grad_dtype=grad_dtype, fuse_t=fuse_t, device=dev)
+    ps.set_option(P.PS_OPT_OVERLAP_LAUNCH, 1)
+    ps.bind_staging(2 * c * fuse_t)
+    ps.init_weights(w0.to(dev))
+    w_host = torch.empty(n_el).pin_memory()
+    pulled, counts, ready = {}, {}, 0
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == 0:
+            pulled[l] = ps.pull_weights()
+            assert ref.pull(l) == pulled[l]
+            continue
+        b = counts.get(l, 0); counts[l] = b + 1
+        g = G.gradient(33, l, b, n_el, 1e-3, dtype=tdt).pin_memory()
+        ref.push(l, as_reference_grad(g))
+        ready += ps.push_gradient(l, g, pulled[l])           # host tensor: cudaMemcpyAsync into a staging slot
+        if ready >= fuse_t:
+            ready -= ps.apply_update()
+            ps.pull_weights(w_host, non_blocking=True)       # the read-back of the e2e leg, overlapping the next uploads
+    ps.flush(); ps.synchronize()
+    assert ps.get_option(P.PS_OPT_LAUNCHES_VECTOR) == pushes // c // fuse_t
+    assert np.array_equal(ps.w.cpu().numpy(), ref.state()[0].astype(np.float32))
+    assert np.array_equal(ps.v.cpu().numpy(), ref.state()[1].astype(np.float32))
+    assert np.array_equal(w_host.numpy(), ps.w.cpu().numpy())
+    assert_logs_equal(ps.update_log(), ref.log())
+    ps.destroy()
 
 
 @pytest.mark.parametrize("grad_dtype,fuse_t,n_el,misalign", [
@@ -328,6 +526,16 @@ def test_contiguous_shards_need_no_synchronisation():
     for _, _, sh in shards:
         assert sh.timestamps() == whole.timestamps()
         assert np.array_equal(sh.update_log(), whole.update_log())
+    # and both are what the reference computes on the whole vector
+    from tests.gpu_harness import as_reference_grad, assert_logs_equal
+    from tests.helpers import replay_reference
+    ref = R.ReferencePS(n_el, lam, n, 0.02, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.cpu().numpy())
+    replay_reference(ref, kinds, learners, lambda l, p: as_reference_grad(G.gradient(14, l, p, n_el, 1e-3, device=dev)))
+    assert np.array_equal(wbuf.cpu().numpy(), ref.state()[0].astype(np.float32))
+    assert np.array_equal(vbuf.cpu().numpy(), ref.state()[1].astype(np.float32))
+    assert_logs_equal(whole.update_log(), ref.log())
+    for _, _, sh in shards:
         sh.destroy()
     whole.destroy()
 
@@ -535,6 +743,8 @@ def test_null_and_misaligned_gradient_pointers_are_rejected():
     assert P.ps_push_gradient(ps._h, 0, None, 0) == P.PS_ERR_INVALID_ARG
     g = torch.ones(66, device=dev)
     assert P.ps_push_gradient(ps._h, 0, g.data_ptr() + 2, 0) == P.PS_ERR_INVALID_ARG
+    host = torch.ones(64)
+    assert P.ps_push_gradient_host(ps._h, 0, host.data_ptr(), 0) == P.PS_ERR_NO_STATE     # no staging slots bound
     assert ps.timestamps() == (0, 0)
     ps.destroy()
 
@@ -591,6 +801,88 @@ def test_learners_write_into_server_owned_slots():
         out.append((ps.w.cpu().numpy().copy(), ps.v.cpu().numpy().copy()))
         ps.destroy()
     assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
+    ref = R.ReferencePS(n_el, lam, 1, 0.02, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    for u in range(5):
+        for l in range(lam):
+            ref.pull(l)
+        for l in range(lam):
+            ref.push(l, G.gradient(41, l, u, n_el, 1e-3).numpy())
+    assert np.array_equal(out[1][0], ref.state()[0].astype(np.float32))
+    assert np.array_equal(out[1][1], ref.state()[1].astype(np.float32))
+
+
+@pytest.mark.parametrize("overlap", [0, 1])
+def test_learner_fills_recycled_slots_from_its_own_stream(overlap):
+    """A learner with its own stream and its own kernels writes gradients straight into receive slots.  With
+    only c + 1 slots every slot is recycled update after update, so a write can meet the update kernel that is still
+    reading the slot's previous gradient unless the learner's stream waits for that kernel (ps_slot_wait),
+    and the update must wait for the learner's kernels (ps_slot_written).  PS_OPT_OVERLAP_LAUNCH is on in
+    one variant: launches that consume learner-written slots must not fetch their gradients early."""
+    from tests.gpu_harness import as_reference_grad
+    dev = torch.device("cuda", 0)
+    n_el, lam = 4_000_001, 2
+    updates = 8                                              # 16 pushes through 3 slots: 5+ generations each
+    w0 = G.initial_weights(layouts.flat(n_el), 43)
+    ref = R.ReferencePS(n_el, lam, 1, 0.02, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    ps = P.ParameterServer(n_el, lam, 1, 0.02, 0.9, 5e-4, device=dev)
+    ps.set_option(P.PS_OPT_OVERLAP_LAUNCH, overlap)
+    ps.bind_staging(lam + 1)
+    ps.init_weights(w0.to(dev))
+    learner_stream = torch.cuda.Stream(dev)
+    seen = set()
+    for u in range(updates):
+        ts = ps.pull_weights()
+        for l in range(lam):
+            assert ref.pull(l) == ts
+        for l in range(lam):
+            sid, view = ps.acquire_slot()
+            seen.add(sid)
+            ps.slot_wait(sid, learner_stream)                # after the kernel that read this slot last
+            with torch.cuda.stream(learner_stream):
+                G.gradient(43, l, u, n_el, 1e-3, device=dev, out=view)      # a chain of the learner's kernels
+            ps.slot_written(sid, learner_stream)             # the server's stream waits for them
+            fired = ps.push_slot(l, sid, ts)
+            ref.push(l, G.gradient(43, l, u, n_el, 1e-3).numpy())
+        assert fired and ps.apply_update() == 1              # no host synchronisation anywhere in the loop
+    ps.synchronize()
+    learner_stream.synchronize()
+    assert lam <= len(seen) <= lam + 1                       # the pool hands back the slot freed last: each one
+                                                             # is rewritten right behind the kernel that read it
+    assert np.array_equal(ps.w.cpu().numpy(), ref.state()[0].astype(np.float32))
+    assert np.array_equal(ps.v.cpu().numpy(), ref.state()[1].astype(np.float32))
+    ps.destroy()
+
+
+def test_stream_change_orders_after_work_on_the_old_stream():
+    """Updates enqueued on the first stream finish before anything enqueued after PS_OPT_STREAM moves the
+    server to another stream; weights and momentum overlapping in memory are refused."""
+    from tests.gpu_harness import as_reference_grad
+    dev = torch.device("cuda", 0)
+    n_el = 3_000_001
+    w0 = G.initial_weights(layouts.flat(n_el), 47)
+    ref = R.ReferencePS(n_el, 1, 1, 0.05, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    ps = P.ParameterServer(n_el, 1, 1, 0.05, 0.9, 5e-4, device=dev)
+    ps.init_weights(w0.to(dev))
+    grads = [G.gradient(47, 0, u, n_el, 1e-3, device=dev) for u in range(8)]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    for u in range(8):
+        ps.set_option(P.PS_OPT_STREAM, streams[u % 2].cuda_stream)          # hop between two streams, no host sync
+        ref.pull(0)
+        ref.push(0, as_reference_grad(grads[u]))
+        ps.push_gradient(0, grads[u], ps.pull_weights())
+        assert ps.apply_update() == 1
+    ps.synchronize()
+    torch.cuda.synchronize()
+    assert np.array_equal(ps.w.cpu().numpy(), ref.state()[0].astype(np.float32))
+    assert np.array_equal(ps.v.cpu().numpy(), ref.state()[1].astype(np.float32))
+    ps.destroy()
+    buf = torch.zeros(100, device=dev)
+    with pytest.raises(P.SoftsyncError):
+        P.ParameterServer(64, 1, 1, 0.1, device=dev, state=(buf[:64], buf[32:96]))
 
 
 def test_staging_slots_run_out():

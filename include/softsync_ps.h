@@ -51,8 +51,10 @@ enum ps_status {
     PS_ERR_NO_STATE = -8,                 /* weights/momentum (or staging slots) not bound yet */
     PS_ERR_LOG_EVICTED = -9,              /* requested log range is no longer (or not yet) held */
     PS_ERR_BARRIER = -10,                 /* hardsync: this learner has already contributed to the current round */
-    PS_ERR_DEVICE_WAIT = -11              /* a bounded wait inside an update kernel ran out (PS_KERNEL_BULK); theta and v
+    PS_ERR_DEVICE_WAIT = -11,             /* a bounded wait inside an update kernel ran out (PS_KERNEL_BULK); theta and v
                                            * are partly updated and must be re-initialised; see ps_kernel_status */
+    PS_ERR_STATIC_LIMIT = -12             /* ps_fused_update_static: more blocks than PS_STATIC_MAX_BLOCKS or more
+                                           * gradients than PS_STATIC_MAX_GRADS: the fixed status area cannot hold it */
 };
 
 enum ps_grad_dtype { PS_GRAD_FP32 = 0, PS_GRAD_BF16 = 1 };
@@ -79,7 +81,7 @@ enum ps_option {
                                            * memory); 0 = chosen from the launch's gradient count (default) */
     PS_OPT_BULK_STAGES = 17,              /* PS_KERNEL_BULK: tiles in flight per block, 2..8 (default 4) */
     PS_OPT_BULK_WAIT_LIMIT = 18,          /* PS_KERNEL_BULK: polls of a copy barrier before the kernel gives up
-                                           * (default 2^22, about a second; at least 16) */
+                                           * (default 2^20, about a second; at least 16) */
     PS_OPT_BULK_SELFTEST = 19             /* PS_KERNEL_BULK, diagnostics: 1 makes block 0 of the NEXT launch announce 16
                                            * bytes more than it copies for its first tile, so that tile's wait runs out;
                                            * the launch then ends with PS_ERR_DEVICE_WAIT recorded.  Resets to 0. */
@@ -318,6 +320,47 @@ int ps_kernel_time(ps_t *ps, double *total_ms, int64_t *launches);
 int ps_last_cuda_error(ps_t *ps);
 
 const char *ps_status_string(int status);
+
+/* One fused update without any allocation.  The paper has no counterpart: this entry point exists for
+ * callers that must not allocate while they run.  Examples: a learner framework whose caching allocator owns
+ * all device memory, so that a cudaMalloc or cudaHostAlloc made behind its back can fail or fragment its
+ * pool; a training loop whose steady state has to stay free of calls that synchronise the device, which
+ * allocation calls do; code that runs where allocation is not permitted at all.  The ordinary path cannot
+ * promise that: ps_create allocates host memory, and the first PS_KERNEL_BULK launch of a handle calls
+ * cudaHostAlloc for the status record its kernel reports through.
+ *
+ * What it does: one weight update (Eq. 2 with momentum and decay, the arithmetic of ps_apply_update for one
+ * group) by the shared-memory staged kernel of PS_KERNEL_BULK, with no handle and no protocol state:
+ *     acc = scales[0] g_0 + ... + scales[c-1] g_{c-1};  v = momentum * v + (acc + decay * theta);  theta -= v
+ * w_dev, v_dev: num_params fp32 each, device memory, read and written.  grads_dev: HOST array of c DEVICE
+ * pointers to num_params values of grad_dtype (ps_grad_dtype) each, read only.  scales_host: HOST array of c
+ * fp32 scales (the caller applies Eq. 3 and the 1/c of Eq. 2 itself).  Every device pointer must be 16-byte
+ * aligned and belong to the current device.  The caller owns every buffer; nothing is kept after the call.
+ * blocks: 0 lets the library choose (two per SM, fewer for short vectors); a positive value caps the grid,
+ * for a server that shares its GPU with learners' kernels.  stream: a cudaStream_t; the work is enqueued
+ * there and the call returns at once unless blocks_gave_up != NULL.
+ *
+ * Scratch memory: the kernel reports a copy wait that ran out in a status record, one per block.  Here the
+ * records are a fixed array of PS_STATIC_MAX_BLOCKS entries (16 KiB) in the library's static device memory,
+ * which every GPU that loads the library holds until the process exits.  A launch that would need more
+ * blocks, or c > PS_STATIC_MAX_GRADS, is refused with PS_ERR_STATIC_LIMIT and does nothing.  All calls on
+ * one device share the array and it keeps the previous call's contents: every call clears the records it
+ * is about to use (a memset enqueued on `stream` before the kernel), so calls whose device work overlaps,
+ * on different streams or from different threads, race on the records and must be serialised by the caller.
+ *
+ * blocks_gave_up != NULL: the call waits for `stream`, reads the records back and stores how many blocks
+ * gave up (0: the update is complete; otherwise theta and v are partly updated).  NULL: nothing is read.
+ *
+ * The first call on each device looks the array's device address up and raises the kernel's shared-memory
+ * limit; make that first call outside any stream capture.  No call of this function uses cudaMalloc,
+ * cudaFree, cudaHostAlloc or any other allocating routine.
+ * Returns PS_OK, PS_ERR_INVALID_ARG, PS_ERR_STATIC_LIMIT or PS_ERR_CUDA. */
+#define PS_STATIC_MAX_BLOCKS 1024
+#define PS_STATIC_MAX_GRADS 16
+int ps_fused_update_static(float *w_dev, float *v_dev, int64_t num_params,
+                           const void *const *grads_dev, const float *scales_host, int c,
+                           float decay, float momentum, int grad_dtype,
+                           int blocks, void *stream, int *blocks_gave_up);
 
 #ifdef __cplusplus
 }

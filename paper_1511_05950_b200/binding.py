@@ -23,7 +23,8 @@ PS_MOD_CONSTANT, PS_MOD_INV_STALENESS, PS_MOD_EXP_STALENESS = 0, 1, 2
 PS_OK, PS_READY = 0, 1
 PS_ERR_INVALID_ARG, PS_ERR_BAD_LEARNER, PS_ERR_BAD_TIMESTAMP, PS_ERR_NOT_READY = -1, -2, -3, -4
 PS_ERR_QUEUE_FULL, PS_ERR_CUDA, PS_ERR_NOMEM, PS_ERR_NO_STATE, PS_ERR_LOG_EVICTED, PS_ERR_BARRIER = -5, -6, -7, -8, -9, -10
-PS_ERR_DEVICE_WAIT = -11
+PS_ERR_DEVICE_WAIT, PS_ERR_STATIC_LIMIT = -11, -12
+PS_STATIC_MAX_BLOCKS, PS_STATIC_MAX_GRADS = 1024, 16
 PS_GRAD_FP32, PS_GRAD_BF16 = 0, 1
 (PS_OPT_GRAD_DTYPE, PS_OPT_FUSE_T, PS_OPT_STREAM, PS_OPT_QUEUE_GROUPS, PS_OPT_LOG_UPDATES,
  PS_OPT_TIMING, PS_OPT_KERNEL, PS_OPT_BLOCK_THREADS, PS_OPT_OVERLAP_LAUNCH, PS_OPT_PROTOCOL,
@@ -50,6 +51,7 @@ EXPORTS = (
     "ps_slot_wait", "ps_slot_written", "ps_kernel_status", "ps_pull_weights", "ps_pull_weights_host", "ps_pull_weights_host_async",
     "ps_push_gradient", "ps_push_gradient_host", "ps_acquire_slot", "ps_push_slot", "ps_release_slot", "ps_apply_update", "ps_flush", "ps_synchronize",
     "ps_get_update_log", "ps_peek_state", "ps_export_state", "ps_import_state", "ps_kernel_time", "ps_last_cuda_error", "ps_status_string",
+    "ps_fused_update_static",
 )
 
 
@@ -101,6 +103,7 @@ def _load() -> C.CDLL:
         "ps_kernel_time": [vp, C.POINTER(C.c_double), C.POINTER(i64)],
         "ps_last_cuda_error": [vp],
         "ps_status_string": [i32],
+        "ps_fused_update_static": [vp, vp, i64, C.POINTER(vp), C.POINTER(f32), i32, f32, f32, i32, i32, vp, C.POINTER(i32)],
     }
     for name, argtypes in sig.items():
         fn = getattr(L, name)
@@ -145,6 +148,7 @@ ps_kernel_time = lib.ps_kernel_time
 ps_export_state = lib.ps_export_state
 ps_import_state = lib.ps_import_state
 ps_last_cuda_error = lib.ps_last_cuda_error
+ps_fused_update_static = lib.ps_fused_update_static
 
 
 def status_string(status: int) -> str:
@@ -179,6 +183,35 @@ def require_tensor(t: torch.Tensor, dtype: torch.dtype, count: int, what: str, o
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
     return None if t is None else t.data_ptr()
+
+
+def fused_update_static(w: torch.Tensor, v: torch.Tensor, grads, scales, decay: float, momentum: float,
+                        blocks: int = 0, read_status: bool = True) -> int:
+    """ps_fused_update_static: one weight update from `grads` (a list of c device tensors, fp32 or bf16)
+    with the given per-gradient scales, for callers that may not allocate device or pinned memory while
+    they run (the kernel's status records sit in the library's static device memory).  Marshals the
+    arguments and nothing else; the work goes to torch's current stream on w's device.  Returns how many
+    blocks gave up on a copy wait (0: complete) when read_status is set, which waits for the stream."""
+    n = w.numel()
+    require_tensor(w, torch.float32, n, "weights", on_gpu=True)
+    require_tensor(v, torch.float32, n, "momentum", on_gpu=True, device=w.device)
+    if len(grads) != len(scales) or not grads:
+        raise ValueError("one scale per gradient, at least one gradient")
+    gdt = grads[0].dtype
+    if gdt not in (torch.float32, torch.bfloat16):
+        raise TypeError("gradients must be fp32 or bf16")
+    for g in grads:
+        require_tensor(g, gdt, n, "gradient", on_gpu=True, device=w.device)
+    ptrs = (C.c_void_p * len(grads))(*[g.data_ptr() for g in grads])
+    sc = (C.c_float * len(grads))(*[float(x) for x in scales])
+    gave_up = C.c_int(0)
+    with torch.cuda.device(w.device):
+        stream = torch.cuda.current_stream(w.device).cuda_stream
+        _check(ps_fused_update_static(w.data_ptr(), v.data_ptr(), n, ptrs, sc, len(grads), decay, momentum,
+                                      PS_GRAD_BF16 if gdt == torch.bfloat16 else PS_GRAD_FP32, blocks,
+                                      C.c_void_p(stream), C.byref(gave_up) if read_status else None),
+               "ps_fused_update_static")
+    return gave_up.value
 
 
 class ParameterServer:

@@ -1101,8 +1101,131 @@ const char *ps_status_string(int status)
     case PS_ERR_LOG_EVICTED: return "log range not held";
     case PS_ERR_BARRIER: return "hardsync: learner already contributed to this round";
     case PS_ERR_DEVICE_WAIT: return "an update kernel gave up on a bounded wait; re-initialise the weights";
+    case PS_ERR_STATIC_LIMIT: return "more blocks or gradients than the static status area of ps_fused_update_static holds";
     default: return status > 1 ? "updates applied" : "unknown status";
     }
 }
 
 }  // extern "C"
+
+// =====================================================================================
+// ps_fused_update_static: one update by the bulk-copy kernel for callers that must not
+// allocate.  The kernel's status records live in static device memory instead of memory
+// obtained at run time.
+// =====================================================================================
+namespace {
+
+// One record per block of the largest grid the entry point accepts.  In host code this name is only a
+// stand-in for the symbol: the address a kernel can use comes from cudaGetSymbolAddress, per device.
+static __device__ __align__(256) BulkStatus g_static_records[PS_STATIC_MAX_BLOCKS];
+
+constexpr int kStaticMaxDevices = 64;
+constexpr int kStaticStages = 4;
+constexpr int kStaticWaitLimit = 1 << 20;
+
+struct StaticSetup {
+    bool done = false;
+    BulkStatus *records = nullptr;     // device address of g_static_records on this device
+    int sm_count = 0;
+};
+StaticSetup g_static_setup[kStaticMaxDevices];
+std::mutex g_static_mutex;
+
+using StaticParams = LaunchParams<kHead, 1>;
+
+template <typename GT>
+auto static_kernel() { return softsync::softsync_update_bulk_kernel<GT, false, kHead, 1, true>; }
+
+// First use on a device: the device address of the record array and the kernel's shared-memory opt-in.
+cudaError_t static_setup(int device, StaticSetup **out)
+{
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticSetup &st = g_static_setup[device];
+    if (!st.done) {
+        BulkStatus *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_records);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(static_kernel<GradFp32>(), cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(static_kernel<GradBf16>(), cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        if (e != cudaSuccess) return e;
+        st.records = ptr;
+        st.done = true;
+    }
+    *out = &st;
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int ps_fused_update_static(float *w_dev, float *v_dev, int64_t num_params,
+                                      const void *const *grads_dev, const float *scales_host, int c,
+                                      float decay, float momentum, int grad_dtype,
+                                      int blocks, void *stream, int *blocks_gave_up)
+{
+  try {
+    if (num_params < 0 || c < 1 || blocks < 0) return PS_ERR_INVALID_ARG;
+    if (grad_dtype != PS_GRAD_FP32 && grad_dtype != PS_GRAD_BF16) return PS_ERR_INVALID_ARG;
+    if (c > PS_STATIC_MAX_GRADS || blocks > PS_STATIC_MAX_BLOCKS) return PS_ERR_STATIC_LIMIT;
+    if (!grads_dev || !scales_host) return PS_ERR_INVALID_ARG;
+    if (blocks_gave_up) *blocks_gave_up = 0;
+    if (num_params == 0) return PS_OK;
+    if (!w_dev || !v_dev || w_dev == v_dev || !aligned16(w_dev) || !aligned16(v_dev)) return PS_ERR_INVALID_ARG;
+    for (int l = 0; l < c; ++l)
+        if (!grads_dev[l] || !aligned16(grads_dev[l])) return PS_ERR_INVALID_ARG;
+
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kStaticMaxDevices) return PS_ERR_CUDA;
+    StaticSetup *setup = nullptr;
+    if (static_setup(device, &setup) != cudaSuccess) return PS_ERR_CUDA;
+
+    StaticParams p;
+    p.w = w_dev; p.v = v_dev; p.n = num_params;
+    p.momentum = momentum; p.T = 1; p.c = c;
+    p.overlap = 0; p.reverse = 0; p.mirror = nullptr;
+    p.layers.count = 0;
+    p.d[0] = decay;
+    for (int l = 0; l < c; ++l) { p.s[l] = scales_host[l]; p.g[l] = grads_dev[l]; }
+
+    // the tile rule of the PS_KERNEL_BULK default: the largest power of two whose stages leave room for two blocks per SM
+    const int gb = grad_dtype == PS_GRAD_BF16 ? 2 : 4;
+    const size_t per_elem = 8 + static_cast<size_t>(c) * gb;
+    int tile = 8192;
+    while (tile > 256 && static_cast<size_t>(kStaticStages) * tile * per_elem > 100 * 1024) tile >>= 1;
+    const size_t smem = static_cast<size_t>(kStaticStages) * tile * per_elem;
+
+    BulkPlan plan;
+    plan.tile_elems = tile;
+    plan.ntiles = num_params / tile;
+    plan.stages = kStaticStages;
+    plan.wait_limit = kStaticWaitLimit;
+    plan.selftest = 0;
+    plan.status = setup->records;
+    long long grid = std::max<long long>(1, std::min<long long>(plan.ntiles, 2ll * setup->sm_count));
+    if (blocks > 0) grid = std::min<long long>(grid, blocks);
+    if (grid > PS_STATIC_MAX_BLOCKS) return PS_ERR_STATIC_LIMIT;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array still holds what the previous call left: clear the records this grid will use
+    if (cudaMemsetAsync(setup->records, 0, static_cast<size_t>(grid) * sizeof(BulkStatus), st) != cudaSuccess) return PS_ERR_CUDA;
+    const dim3 g(static_cast<unsigned>(grid)), b(kBulkThreads);
+    if (grad_dtype == PS_GRAD_BF16)
+        softsync::softsync_update_bulk_kernel<GradBf16, false, kHead, 1, true><<<g, b, smem, st>>>(p, plan);
+    else
+        softsync::softsync_update_bulk_kernel<GradFp32, false, kHead, 1, true><<<g, b, smem, st>>>(p, plan);
+    if (cudaGetLastError() != cudaSuccess) return PS_ERR_CUDA;
+
+    if (blocks_gave_up) {
+        BulkStatus seen[PS_STATIC_MAX_BLOCKS];
+        if (cudaStreamSynchronize(st) != cudaSuccess) return PS_ERR_CUDA;
+        if (cudaMemcpy(seen, setup->records, static_cast<size_t>(grid) * sizeof(BulkStatus), cudaMemcpyDeviceToHost) != cudaSuccess)
+            return PS_ERR_CUDA;
+        int gave_up = 0;
+        for (long long k = 0; k < grid; ++k) gave_up += seen[k].code != 0;
+        *blocks_gave_up = gave_up;
+    }
+    return PS_OK;
+  } PS_CATCH_ALL
+}

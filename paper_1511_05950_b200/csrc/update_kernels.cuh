@@ -384,7 +384,9 @@ __device__ __forceinline__ void update_from_stage(const Params &p, const unsigne
     if (p.mirror) store_mirror<VEC>(p.mirror + first, f.w);
 }
 
-template <typename GT, bool LAYERS, int MAXE, int MAXSEG>
+// BLOCK_RECORDS: plan.status is an array with one record per block of the grid (each block that gives up
+// writes its own) instead of one record shared by the launch.
+template <typename GT, bool LAYERS, int MAXE, int MAXSEG, bool BLOCK_RECORDS = false>
 __global__ void softsync_update_bulk_kernel(const __grid_constant__ LaunchParams<MAXE, MAXSEG> p,
                                             const __grid_constant__ BulkPlan plan)
 {
@@ -486,7 +488,7 @@ __global__ void softsync_update_bulk_kernel(const __grid_constant__ LaunchParams
         const long long issued = (k + S < mine) ? k + S : mine;     // tiles k .. issued-1 were issued and not consumed
         for (long long j = k; j < issued; ++j)
             mbar_wait_bounded(smem_addr(&full[j % S]), static_cast<unsigned>((j / S) & 1), plan.wait_limit);
-        volatile BulkStatus *st = plan.status;
+        volatile BulkStatus *st = BLOCK_RECORDS ? plan.status + b : plan.status;
         st->block = static_cast<int>(b);
         st->stage = static_cast<int>(k % S);
         st->tile = static_cast<int>(k);

@@ -150,7 +150,7 @@ constexpr int kBulkThreads = 256;
 template <bool LAYERS> constexpr int seg_capacity() { return LAYERS ? PS_MAX_LAYERS : 1; }
 template <int MAXE, bool LAYERS> using Params = LaunchParams<MAXE, seg_capacity<LAYERS>()>;
 
-template <typename GT, int VEC, int EC, bool MORE, bool LAYERS, int MAXE>
+template <typename GT, int VEC, int EC, bool MORE, bool LAYERS, int MAXE, int CT = 0>
 cudaError_t launch_variant(const Params<MAXE, LAYERS> &p, int blocks, int threads, cudaStream_t stream)
 {
     cudaLaunchConfig_t cfg = {};
@@ -162,7 +162,7 @@ cudaError_t launch_variant(const Params<MAXE, LAYERS> &p, int blocks, int thread
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = p.overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, softsync::softsync_update_kernel<GT, VEC, EC, MORE, kChunk, LAYERS, MAXE, seg_capacity<LAYERS>()>, p);
+    return cudaLaunchKernelEx(&cfg, softsync::softsync_update_kernel<GT, VEC, EC, MORE, kChunk, LAYERS, MAXE, seg_capacity<LAYERS>(), CT>, p);
 }
 
 // E = T*c <= HEAD: the straight-line instantiation with exactly E loads up front.
@@ -172,7 +172,12 @@ cudaError_t launch_exact(int E, const Params<MAXE, LAYERS> &p, int blocks, int t
     if constexpr (EC == 0) {
         return cudaErrorInvalidValue;
     } else {
-        if (E == EC) return launch_variant<GT, VEC, EC, false, LAYERS, MAXE>(p, blocks, threads, stream);
+        if (E == EC) {
+            // c = 1 (every gradient its own update, the fused asynchronous case) has its own instantiation
+            if constexpr (!LAYERS)
+                if (p.c == 1) return launch_variant<GT, VEC, EC, false, LAYERS, MAXE, 1>(p, blocks, threads, stream);
+            return launch_variant<GT, VEC, EC, false, LAYERS, MAXE>(p, blocks, threads, stream);
+        }
         return launch_exact<GT, VEC, HEAD, LAYERS, MAXE, EC - 1>(E, p, blocks, threads, stream);
     }
 }

@@ -174,33 +174,85 @@ __device__ __forceinline__ int find_layer(const LayerTable<MAXSEG> &tab, long lo
     return lo;
 }
 
-// Adds gradient entry e (already in registers) to the fragment; when it is the
-// last of its group, performs that group's weight update.  Branches are uniform
-// across the grid (they depend on e and c only).
-template <typename GT, int VEC, bool LAYERS, typename Params>
-__device__ __forceinline__ void consume(const Params &p, Fragment<VEC> &f, const Raw<GT, VEC> &r, int e)
+// Packed fp32 pairs (sm_100 f32x2).  One packed multiply or subtract rounds each half exactly like its
+// scalar form and costs one issue slot for two elements.  Only multiplies whose results feed SCALAR adds, and
+// subtracts whose operands are not products, are packed: a packed multiply feeding a packed add is contracted
+// into a fused multiply-add by ptxas 12.9 (single rounding), which the arithmetic contract forbids.
+__device__ __forceinline__ void mul_pair(float &x0, float &x1, float a, float b0, float b1)
 {
-    float g[VEC];
-    widen(r, g);
-    const float s = p.s[e];
-    if (f.l == 0) {
-#pragma unroll
-        for (int j = 0; j < VEC; ++j) f.acc[j] = __fmul_rn(s, g[j]);
+    unsigned long long A, B, R;
+    asm("mov.b64 %0, {%1,%1};" : "=l"(A) : "f"(a));
+    asm("mov.b64 %0, {%1,%2};" : "=l"(B) : "f"(b0), "f"(b1));
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(R) : "l"(A), "l"(B));
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(x0), "=f"(x1) : "l"(R));
+}
+__device__ __forceinline__ void sub_pair(float &x0, float &x1, float a0, float a1, float b0, float b1)
+{
+    unsigned long long A, B, R;
+    asm("mov.b64 %0, {%1,%2};" : "=l"(A) : "f"(a0), "f"(a1));
+    asm("mov.b64 %0, {%1,%2};" : "=l"(B) : "f"(b0), "f"(b1));
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(R) : "l"(A), "l"(B));
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(x0), "=f"(x1) : "l"(R));
+}
+// x[j] = a * y[j], every product rounded once
+template <int VEC>
+__device__ __forceinline__ void scale(float (&x)[VEC], float a, const float (&y)[VEC])
+{
+    if constexpr (VEC == 4) {
+        mul_pair(x[0], x[1], a, y[0], y[1]);
+        mul_pair(x[2], x[3], a, y[2], y[3]);
     } else {
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) f.acc[j] = __fadd_rn(f.acc[j], __fmul_rn(s, g[j]));
+        for (int j = 0; j < VEC; ++j) x[j] = __fmul_rn(a, y[j]);
     }
-    if (++f.l == p.c) {                                  // group complete: one weight update
-        float d = p.d[f.t++];
-        const float m = p.momentum;
-        f.l = 0;
-        if constexpr (LAYERS) d = __fmul_rn(f.dm, d);
+}
+
+// Adds gradient entry e (already in registers) to the fragment; when it is the
+// last of its group, performs that group's weight update.  Branches are uniform
+// across the grid (they depend on e and c only).  CT = 1: the launch has c = 1, known at
+// compile time: every entry is a group of its own, entry e is group e, and the position
+// counters and their branches disappear (they are a quarter of the instructions of a fused
+// bf16 pass otherwise).  CT = 0: c is read from the launch parameters.
+template <typename GT, int VEC, bool LAYERS, int CT = 0, typename Params>
+__device__ __forceinline__ void consume(const Params &p, Fragment<VEC> &f, const Raw<GT, VEC> &r, int e)
+{
+    float g[VEC], prod[VEC];
+    widen(r, g);
+    scale<VEC>(prod, p.s[e], g);
+    bool complete = true;
+    float d;
+    if constexpr (CT == 1) {
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) {
-            float tt = __fadd_rn(f.acc[j], __fmul_rn(d, f.w[j]));
-            if constexpr (LAYERS) tt = __fmul_rn(f.lm, tt);
-            f.v[j] = __fadd_rn(__fmul_rn(m, f.v[j]), tt);
-            f.w[j] = __fsub_rn(f.w[j], f.v[j]);
+        for (int j = 0; j < VEC; ++j) f.acc[j] = prod[j];
+        d = p.d[e];
+    } else {
+        if (f.l == 0) {
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) f.acc[j] = prod[j];
+        } else {
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) f.acc[j] = __fadd_rn(f.acc[j], prod[j]);
+        }
+        complete = ++f.l == p.c;
+        if (complete) { d = p.d[f.t++]; f.l = 0; }
+    }
+    if (complete) {                                      // group complete: one weight update
+        const float m = p.momentum;
+        if constexpr (LAYERS) d = __fmul_rn(f.dm, d);
+        float dw[VEC], mv[VEC], tt[VEC];
+        scale<VEC>(dw, d, f.w);
+        scale<VEC>(mv, m, f.v);
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) tt[j] = __fadd_rn(f.acc[j], dw[j]);
+        if constexpr (LAYERS) scale<VEC>(tt, f.lm, tt);
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) f.v[j] = __fadd_rn(mv[j], tt[j]);
+        if constexpr (VEC == 4) {
+            sub_pair(f.w[0], f.w[1], f.w[0], f.w[1], f.v[0], f.v[1]);
+            sub_pair(f.w[2], f.w[3], f.w[2], f.w[3], f.v[2], f.v[3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) f.w[j] = __fsub_rn(f.w[j], f.v[j]);
         }
     }
 }
@@ -211,7 +263,7 @@ __device__ __forceinline__ void consume(const Params &p, Fragment<VEC> &f, const
 // flight.  MORE = false: the launch has exactly EC entries and the code is
 // straight-line (no spare registers held for a loop that never runs).
 // MORE = true: entries beyond EC follow in chunks of K loads, the last few one by one.
-template <typename GT, int VEC, int EC, bool MORE, int K, bool LAYERS, typename Params>
+template <typename GT, int VEC, int EC, bool MORE, int K, bool LAYERS, int CT = 0, typename Params>
 __device__ __forceinline__ void update_fragment(const Params &p, long long i, long long first, float lm, float dm)
 {
     Fragment<VEC> f;
@@ -223,8 +275,9 @@ __device__ __forceinline__ void update_fragment(const Params &p, long long i, lo
     load_state<VEC>(p.v + first, f.v);
     f.l = 0; f.t = 0; f.lm = lm; f.dm = dm;
 #pragma unroll
-    for (int e = 0; e < EC; ++e) consume<GT, VEC, LAYERS>(p, f, head[e], e);
+    for (int e = 0; e < EC; ++e) consume<GT, VEC, LAYERS, CT>(p, f, head[e], e);
     if constexpr (MORE) {
+        static_assert(CT == 0, "the compile-time group size is for straight-line launches only");
         const int E = p.T * p.c;
         int e0 = EC;
         for (; e0 + K <= E; e0 += K) {                   // full chunks: K independent loads, no predicates
@@ -261,10 +314,10 @@ __device__ __forceinline__ void update_element(const Params &p, long long k)
 // (blocks * threads >= n / VEC).  No grid-stride loop: a loop around the fragment
 // makes the compiler keep a second iteration's registers alive and costs a third
 // of the occupancy.  The host guarantees T*c == EC (MORE = false) or T*c > EC
-// (MORE = true).  The (n mod VEC) trailing elements are done one by one by the
-// first threads of the grid.  LAYERS: the fragment's multipliers are looked up once;
+// (MORE = true), and c = 1 when CT = 1 (used without a layer table only).  The (n mod VEC)
+// trailing elements are done one by one by the first threads of the grid.  LAYERS: the fragment's multipliers are looked up once;
 // a fragment that straddles a layer boundary is done element by element.
-template <typename GT, int VEC, int EC, bool MORE, int K, bool LAYERS, int MAXE, int MAXSEG>
+template <typename GT, int VEC, int EC, bool MORE, int K, bool LAYERS, int MAXE, int MAXSEG, int CT = 0>
 __global__ void softsync_update_kernel(const __grid_constant__ LaunchParams<MAXE, MAXSEG> p)
 {
     const long long nfrag = p.n / VEC;
@@ -285,7 +338,7 @@ __global__ void softsync_update_kernel(const __grid_constant__ LaunchParams<MAXE
         } else if constexpr (LAYERS) {
             update_element<GT, K, true>(p, first);
         } else {
-            update_fragment<GT, VEC, EC, MORE, K, false>(p, i, first, 1.f, 1.f);
+            update_fragment<GT, VEC, EC, MORE, K, false, CT>(p, i, first, 1.f, 1.f);
         }
     }
     if constexpr (VEC > 1) {

@@ -190,6 +190,8 @@ def build_server(P, cfg, args, dev, rank, fuse_t):
     ps.set_option(P.PS_OPT_KERNEL, P.binding.KERNELS[args.kernel])
     if args.block_threads:
         ps.set_option(P.PS_OPT_BLOCK_THREADS, args.block_threads)
+    if args.no_zigzag:
+        ps.set_option(P.PS_OPT_ZIGZAG, 0)
     if args.bulk_tile:
         ps.set_option(P.PS_OPT_BULK_TILE, args.bulk_tile)
     if args.bulk_stages:
@@ -360,8 +362,8 @@ def run_ours(args, cfg, rank, world, local_rank):
     kernel_name = {1: "scalar", 2: "vector", 3: "bulk"}.get(facts["last_kernel"], "none")
     traffic, traffic_from = traffic_for(cfg.name, kernel_name, cfg.grad_dtype, cfg.c, fuse_t, args.block_threads,
                                         args.bf16_mirror, args.layer_multipliers)
-    if args.no_overlap and traffic is not None:
-        traffic, traffic_from = None, "the recorded capture used programmatic dependent launches"
+    if (args.no_overlap or args.no_zigzag) and traffic is not None:
+        traffic, traffic_from = None, "the recorded capture used programmatic dependent launches and alternating traversal"
     mid = sorted(reps, key=lambda r: r["ms"])[len(reps) // 2]
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -377,6 +379,7 @@ def run_ours(args, cfg, rank, world, local_rank):
             "bf16_mirror": bool(args.bf16_mirror), "layer_multipliers": bool(args.layer_multipliers),
             "kernel": kernel_name, "kernel_launches": facts["launches"],
             "launch": "ordinary" if args.no_overlap else "programmatic dependent launch (PS_OPT_OVERLAP_LAUNCH=1)",
+            "traversal": "forward" if args.no_zigzag else "alternating direction from launch to launch",
             "parallelism": ("%d contiguous shards of one %d-parameter vector, no data-path collective"
                             % (world, args.total_params)) if args.total_params else
                            ("replicas only (independent servers, no data-path collective)" if world > 1 else "1 GPU"),
@@ -662,6 +665,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="ordinary launches instead of programmatic dependent ones")
+    ap.add_argument("--no-zigzag", action="store_true", help="every launch walks the vector forward (PS_OPT_ZIGZAG=0)")
     ap.add_argument("--bf16-mirror", action="store_true",
                     help="variant: keep a bf16 copy of the weights current in the same pass (+2 bytes per element)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
@@ -712,7 +716,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     result, e2e_detail = run_ours(args, cfg, rank, world, local_rank)
     default_run = (args.workload == "large_softsync" and not args.num_params and not args.total_params
-                   and args.kernel == "auto" and not args.bf16_mirror and not args.layer_multipliers)
+                   and args.kernel == "auto" and not args.bf16_mirror and not args.layer_multipliers
+                   and not args.no_zigzag)
     if default_run and not args.no_second_config:
         result["configs"] = {"large_stale_bf16": second_config(args, rank, world, local_rank)}
     if rank == 0:

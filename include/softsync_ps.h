@@ -68,7 +68,7 @@ enum ps_option {
     PS_OPT_LOG_UPDATES = 5,               /* how many most recent updates the log keeps (default max(1024, 2^20 / c)) */
     PS_OPT_TIMING = 6,                    /* 1: bracket every update kernel with CUDA events (ps_kernel_time) */
     PS_OPT_KERNEL = 7,                    /* ps_kernel_choice (default PS_KERNEL_AUTO) */
-    PS_OPT_BLOCK_THREADS = 8,             /* threads per block: 128, 256 or 512; 0 = default (128; 256 for PS_KERNEL_BULK) */
+    PS_OPT_BLOCK_THREADS = 8,             /* threads per block: 128, 256 or 512; 0 = default (128; 512 for PS_KERNEL_BULK) */
     PS_OPT_OVERLAP_LAUNCH = 9,            /* 1: update kernels are launched as programmatic dependents (see below); default 0 */
     PS_OPT_PROTOCOL = 10,                 /* ps_protocol (default PS_PROTOCOL_SOFTSYNC); only while nothing is pending */
     PS_OPT_GROUP_SIZE = 11,               /* read-only: c = floor(lambda / n) of Eq. 2 */
@@ -77,14 +77,17 @@ enum ps_option {
     PS_OPT_LAUNCHES_VECTOR = 14,          /*            the vector kernel, */
     PS_OPT_LAUNCHES_BULK = 15,            /*            the bulk-copy kernel */
     PS_OPT_BULK_TILE = 16,                /* PS_KERNEL_BULK: elements per shared-memory tile, a power of two in
-                                           * [256, 8192] (halved until the stages of one block fit an SM's shared
-                                           * memory); 0 = chosen from the launch's gradient count (default) */
-    PS_OPT_BULK_STAGES = 17,              /* PS_KERNEL_BULK: tiles in flight per block, 2..8 (default 4) */
+                                           * [256, 8192] (halved until the stages of one block fit 200 KB of an SM's
+                                           * shared memory); 0 = the largest that fits (default) */
+    PS_OPT_BULK_STAGES = 17,              /* PS_KERNEL_BULK: tiles in flight per block, 2..8 (default 2) */
     PS_OPT_BULK_WAIT_LIMIT = 18,          /* PS_KERNEL_BULK: polls of a copy barrier before the kernel gives up
                                            * (default 2^20, about a second; at least 16) */
-    PS_OPT_BULK_SELFTEST = 19             /* PS_KERNEL_BULK, diagnostics: 1 makes block 0 of the NEXT launch announce 16
+    PS_OPT_BULK_SELFTEST = 19,            /* PS_KERNEL_BULK, diagnostics: 1 makes block 0 of the NEXT launch announce 16
                                            * bytes more than it copies for its first tile, so that tile's wait runs out;
                                            * the launch then ends with PS_ERR_DEVICE_WAIT recorded.  Resets to 0. */
+    PS_OPT_ZIGZAG = 20                    /* 1 (default): successive update launches walk the vector in opposite directions,
+                                           * so a launch starts on the part of theta and v the previous one left in
+                                           * the L2; 0: every launch walks forward.  Same bits either way. */
 };
 
 /* PS_OPT_OVERLAP_LAUNCH = 1 lets an update kernel start while the previous kernel on the stream is still
@@ -114,7 +117,8 @@ enum ps_kernel_choice {
                                            * cluster, no multicast).  Needs every pointer 16-byte aligned and at most 16
                                            * gradients per launch (T * c <= 16), else PS_ERR_INVALID_ARG.  Same bits as the
                                            * other kernels.  Never chosen by PS_KERNEL_AUTO: on this element-wise, touch-once
-                                           * pass it measures slower than the register kernel; it exists so that the
+                                           * pass it measures level with the register kernel at best (large tiles, two
+                                           * stages) and is the more restricted of the two; it exists so that the
                                            * comparison can be repeated.  Every barrier wait in it is bounded
                                            * (PS_OPT_BULK_WAIT_LIMIT).  Its first launch allocates 64 bytes of pinned host
                                            * memory for the status record. */
@@ -336,7 +340,7 @@ const char *ps_status_string(int status);
  * pointers to num_params values of grad_dtype (ps_grad_dtype) each, read only.  scales_host: HOST array of c
  * fp32 scales (the caller applies Eq. 3 and the 1/c of Eq. 2 itself).  Every device pointer must be 16-byte
  * aligned and belong to the current device.  The caller owns every buffer; nothing is kept after the call.
- * blocks: 0 lets the library choose (two per SM, fewer for short vectors); a positive value caps the grid,
+ * blocks: 0 lets the library choose (as many as fit the SMs, fewer for short vectors); a positive value caps the grid,
  * for a server that shares its GPU with learners' kernels.  stream: a cudaStream_t; the work is enqueued
  * there and the call returns at once unless blocks_gave_up != NULL.
  *

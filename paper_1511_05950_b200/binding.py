@@ -29,7 +29,7 @@ PS_GRAD_FP32, PS_GRAD_BF16 = 0, 1
 (PS_OPT_GRAD_DTYPE, PS_OPT_FUSE_T, PS_OPT_STREAM, PS_OPT_QUEUE_GROUPS, PS_OPT_LOG_UPDATES,
  PS_OPT_TIMING, PS_OPT_KERNEL, PS_OPT_BLOCK_THREADS, PS_OPT_OVERLAP_LAUNCH, PS_OPT_PROTOCOL,
  PS_OPT_GROUP_SIZE, PS_OPT_LAST_KERNEL, PS_OPT_LAUNCHES_SCALAR, PS_OPT_LAUNCHES_VECTOR, PS_OPT_LAUNCHES_BULK,
- PS_OPT_BULK_TILE, PS_OPT_BULK_STAGES, PS_OPT_BULK_WAIT_LIMIT, PS_OPT_BULK_SELFTEST) = range(1, 20)
+ PS_OPT_BULK_TILE, PS_OPT_BULK_STAGES, PS_OPT_BULK_WAIT_LIMIT, PS_OPT_BULK_SELFTEST, PS_OPT_ZIGZAG) = range(1, 21)
 PS_PROTOCOL_SOFTSYNC, PS_PROTOCOL_HARDSYNC = 0, 1
 PS_KERNEL_AUTO, PS_KERNEL_SCALAR, PS_KERNEL_VECTOR, PS_KERNEL_BULK = 0, 1, 2, 3
 PS_MAX_GROUP, PS_MAX_FUSE_T, PS_MAX_ENTRIES, PS_MAX_LAYERS = 256, 16, 512, 64

@@ -66,9 +66,10 @@ struct ps_ctx {
     int64_t log_updates = 65536;           // set in ps_create: about one million log entries
     int timing = 0, kernel_choice = PS_KERNEL_AUTO, block_threads = 0, overlap_launch = 0;
     int protocol = PS_PROTOCOL_SOFTSYNC;
+    int zigzag = 1;
     int sm_count = 0;
 
-    int bulk_tile = 0, bulk_stages = 4, bulk_wait_limit = 1 << 20, bulk_selftest = 0;
+    int bulk_tile = 0, bulk_stages = 2, bulk_wait_limit = 1 << 20, bulk_selftest = 0;
     BulkStatus *bulk_status = nullptr;     // pinned, device-mapped host memory (allocated by the first bulk launch)
     bool bulk_attr_set[2][2] = {};         // dynamic shared-memory opt-in done, per (dtype, layers) instantiation
 
@@ -145,7 +146,7 @@ bool entry_before(const Entry &a, const Entry &b)
 
 constexpr int kChunk = 8;            // gradient loads in flight per thread beyond the first EC
 constexpr int kHead = 16;            // largest compile-time first chunk of gradient loads
-constexpr int kBulkThreads = 256;
+constexpr int kBulkThreads = 512;
 
 template <bool LAYERS> constexpr int seg_capacity() { return LAYERS ? PS_MAX_LAYERS : 1; }
 template <int MAXE, bool LAYERS> using Params = LaunchParams<MAXE, seg_capacity<LAYERS>()>;
@@ -193,22 +194,37 @@ cudaError_t launch_vector(int E, const Params<MAXE, LAYERS> &p, int blocks, int 
     return launch_variant<GT, VEC, HEAD, true, LAYERS, MAXE>(p, blocks, threads, stream);   // HEAD loads, then chunks
 }
 
-// The bulk-copy kernel: tile and grid sizes from the shared memory one block may take.
+// Launch shape of the bulk-copy kernel.  Measured on the 61 M-element configurations, few large tiles win:
+// two stages whose tiles fill most of an SM's shared memory (one block per SM) run 8-25 % faster than four
+// stages of quarter-size tiles (two blocks per SM), because every tile costs a block-wide barrier and one
+// thread's round of copy instructions.
+struct BulkShape { int tile; size_t smem; int threads; int blocks_per_sm; };
+
+BulkShape bulk_shape(int entries, int grad_bytes, int stages, int tile_option, int threads_option)
+{
+    const size_t per_elem = 8 + static_cast<size_t>(entries) * grad_bytes;
+    const size_t limit = 200 * 1024;                     // of the 227 KB one block may take
+    int tile = tile_option ? tile_option : 8192;         // halved until the stages of one block fit
+    while (tile > 256 && static_cast<size_t>(stages) * tile * per_elem > limit) tile >>= 1;
+    BulkShape sh;
+    sh.tile = tile;
+    sh.smem = static_cast<size_t>(stages) * tile * per_elem;
+    sh.threads = threads_option ? threads_option : kBulkThreads;
+    const size_t per_sm = 227 * 1024;
+    const int by_smem = static_cast<int>(std::max<size_t>(1, per_sm / (sh.smem + 1024)));
+    sh.blocks_per_sm = std::max(1, std::min(by_smem, 2048 / sh.threads));
+    return sh;
+}
+
 template <typename GT, bool LAYERS, int MAXE>
 cudaError_t launch_bulk(ps_ctx *ps, const Params<MAXE, LAYERS> &p)
 {
     constexpr int kSeg = seg_capacity<LAYERS>();
     const int gb = ps->grad_dtype == PS_GRAD_BF16 ? 2 : 4;
-    const int E = p.T * p.c;
-    const size_t per_elem = 8 + static_cast<size_t>(E) * gb;
     const int stages = ps->bulk_stages;
-    const size_t budget = 100 * 1024;                    // two blocks per SM
-    // default: the largest tile that leaves room for two blocks per SM; a tile asked for by option is
-    // halved until one block's stages fit the shared memory of an SM
-    int tile = ps->bulk_tile ? ps->bulk_tile : 8192;
-    const size_t limit = ps->bulk_tile ? 200 * 1024 : budget;
-    while (tile > 256 && static_cast<size_t>(stages) * tile * per_elem > limit) tile >>= 1;
-    const size_t smem = static_cast<size_t>(stages) * tile * per_elem;
+    const BulkShape sh = bulk_shape(p.T * p.c, gb, stages, ps->bulk_tile, ps->block_threads);
+    const int tile = sh.tile;
+    const size_t smem = sh.smem;
     if (smem > 220 * 1024) return cudaErrorInvalidConfiguration;
     auto kernel = softsync::softsync_update_bulk_kernel<GT, LAYERS, MAXE, kSeg>;
     bool &attr_set = ps->bulk_attr_set[gb == 2][LAYERS];
@@ -231,11 +247,8 @@ cudaError_t launch_bulk(ps_ctx *ps, const Params<MAXE, LAYERS> &p)
     ps->bulk_selftest = 0;
     cudaError_t e = cudaHostGetDevicePointer(reinterpret_cast<void **>(&plan.status), ps->bulk_status, 0);
     if (e != cudaSuccess) return e;
-    const int threads = ps->block_threads ? ps->block_threads : kBulkThreads;
-    const size_t per_sm = 227 * 1024;
-    const int by_smem = static_cast<int>(std::max<size_t>(1, per_sm / (smem + 1024)));
-    const int per_sm_blocks = std::max(1, std::min(by_smem, 2048 / threads));
-    const long long cap = static_cast<long long>(ps->sm_count) * per_sm_blocks;
+    const int threads = sh.threads;
+    const long long cap = static_cast<long long>(ps->sm_count) * sh.blocks_per_sm;
     const int blocks = static_cast<int>(std::max<long long>(1, std::min<long long>(plan.ntiles, cap)));
 
     cudaLaunchConfig_t cfg = {};
@@ -290,7 +303,7 @@ void build_launch(ps_ctx *ps, int T, Params<MAXE, LAYERS> &p, std::vector<ps_log
     p.w = ps->w; p.v = ps->v; p.n = ps->n;
     p.momentum = ps->momentum; p.T = T; p.c = ps->c;
     p.overlap = ps->overlap_launch;
-    p.reverse = static_cast<int>(ps->launches & 1);      // zig-zag over the vector from launch to launch
+    p.reverse = ps->zigzag ? static_cast<int>(ps->launches & 1) : 0;   // zig-zag over the vector from launch to launch
     p.mirror = ps->mirror;
     p.layers.count = 0;
     if constexpr (LAYERS) {
@@ -701,6 +714,9 @@ int ps_set_option(ps_t *ps, int key, int64_t value)
         case PS_OPT_BLOCK_THREADS:
             if (value != 0 && value != 128 && value != 256 && value != 512) return PS_ERR_INVALID_ARG;
             ps->block_threads = static_cast<int>(value); return PS_OK;
+        case PS_OPT_ZIGZAG:
+            if (value != 0 && value != 1) return PS_ERR_INVALID_ARG;
+            ps->zigzag = static_cast<int>(value); return PS_OK;
         default:
             return PS_ERR_INVALID_ARG;
         }
@@ -731,6 +747,7 @@ int ps_get_option(ps_t *ps, int key, int64_t *value)
         case PS_OPT_BULK_STAGES: *value = ps->bulk_stages; return PS_OK;
         case PS_OPT_BULK_WAIT_LIMIT: *value = ps->bulk_wait_limit; return PS_OK;
         case PS_OPT_BULK_SELFTEST: *value = ps->bulk_selftest; return PS_OK;
+        case PS_OPT_ZIGZAG: *value = ps->zigzag; return PS_OK;
         default: return PS_ERR_INVALID_ARG;
         }
     } PS_CATCH_ALL
@@ -1125,7 +1142,7 @@ namespace {
 static __device__ __align__(256) BulkStatus g_static_records[PS_STATIC_MAX_BLOCKS];
 
 constexpr int kStaticMaxDevices = 64;
-constexpr int kStaticStages = 4;
+constexpr int kStaticStages = 2;
 constexpr int kStaticWaitLimit = 1 << 20;
 
 struct StaticSetup {
@@ -1194,12 +1211,11 @@ extern "C" int ps_fused_update_static(float *w_dev, float *v_dev, int64_t num_pa
     p.d[0] = decay;
     for (int l = 0; l < c; ++l) { p.s[l] = scales_host[l]; p.g[l] = grads_dev[l]; }
 
-    // the tile rule of the PS_KERNEL_BULK default: the largest power of two whose stages leave room for two blocks per SM
+    // the launch shape of the PS_KERNEL_BULK default
     const int gb = grad_dtype == PS_GRAD_BF16 ? 2 : 4;
-    const size_t per_elem = 8 + static_cast<size_t>(c) * gb;
-    int tile = 8192;
-    while (tile > 256 && static_cast<size_t>(kStaticStages) * tile * per_elem > 100 * 1024) tile >>= 1;
-    const size_t smem = static_cast<size_t>(kStaticStages) * tile * per_elem;
+    const BulkShape sh = bulk_shape(c, gb, kStaticStages, 0, 0);
+    const int tile = sh.tile;
+    const size_t smem = sh.smem;
 
     BulkPlan plan;
     plan.tile_elems = tile;
@@ -1208,14 +1224,14 @@ extern "C" int ps_fused_update_static(float *w_dev, float *v_dev, int64_t num_pa
     plan.wait_limit = kStaticWaitLimit;
     plan.selftest = 0;
     plan.status = setup->records;
-    long long grid = std::max<long long>(1, std::min<long long>(plan.ntiles, 2ll * setup->sm_count));
+    long long grid = std::max<long long>(1, std::min<long long>(plan.ntiles, static_cast<long long>(sh.blocks_per_sm) * setup->sm_count));
     if (blocks > 0) grid = std::min<long long>(grid, blocks);
     if (grid > PS_STATIC_MAX_BLOCKS) return PS_ERR_STATIC_LIMIT;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the array still holds what the previous call left: clear the records this grid will use
     if (cudaMemsetAsync(setup->records, 0, static_cast<size_t>(grid) * sizeof(BulkStatus), st) != cudaSuccess) return PS_ERR_CUDA;
-    const dim3 g(static_cast<unsigned>(grid)), b(kBulkThreads);
+    const dim3 g(static_cast<unsigned>(grid)), b(static_cast<unsigned>(sh.threads));
     if (grad_dtype == PS_GRAD_BF16)
         softsync::softsync_update_bulk_kernel<GradBf16, false, kHead, 1, true><<<g, b, smem, st>>>(p, plan);
     else

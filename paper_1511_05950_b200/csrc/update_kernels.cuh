@@ -427,10 +427,20 @@ __device__ __forceinline__ void update_from_stage(const Params &p, const unsigne
 #pragma unroll
     for (int j = 0; j < VEC; ++j) { f.w[j] = ws[li * VEC + j]; f.v[j] = vs[li * VEC + j]; }
     f.l = 0; f.t = 0; f.lm = lm; f.dm = dm;
-    for (int e = 0; e < E; ++e) {
-        Raw<GT, VEC> r;
-        load_raw_shared(r, gs + static_cast<size_t>(e) * tile_elems * GB, li);
-        consume<GT, VEC, LAYERS>(p, f, r, e);
+    if (p.c == 1) {                                      // every entry its own update: no position counters
+#pragma unroll 4
+        for (int e = 0; e < E; ++e) {
+            Raw<GT, VEC> r;
+            load_raw_shared(r, gs + static_cast<size_t>(e) * tile_elems * GB, li);
+            consume<GT, VEC, LAYERS, 1>(p, f, r, e);
+        }
+    } else {
+#pragma unroll 4
+        for (int e = 0; e < E; ++e) {
+            Raw<GT, VEC> r;
+            load_raw_shared(r, gs + static_cast<size_t>(e) * tile_elems * GB, li);
+            consume<GT, VEC, LAYERS>(p, f, r, e);
+        }
     }
     store_state<VEC>(p.w + first, f.w);
     store_state<VEC>(p.v + first, f.v);

@@ -158,3 +158,15 @@ def assert_parity(w, v, log, refs, tol, layout=None):
         assert worst <= tol, "relative L2 error %.3e above %.1e" % (worst, tol)
         return worst
     return 0.0
+
+
+def parity_line(name, elements, updates, compared, w, v, w32, v32, w64, v64):
+    """One row of the parity table (printed by the configuration tests; shown with pytest -s): distance of
+    the GPU state from the fp64 reference, distance of the fp32 reference from the fp64 one (what keeping the
+    state in fp32 costs by itself), and whether GPU and fp32 reference agree bit for bit."""
+    same = bool(np.array_equal(w, np.asarray(w32, np.float32)) and np.array_equal(v, np.asarray(v32, np.float32)))
+    line = "PARITY | %s | %d | %d | %s | %.2e | %.2e | %.2e | %.2e | %s |" % (
+        name, elements, updates, compared, rel_l2(w, w64), rel_l2(v, v64), rel_l2(w32, w64), rel_l2(v32, v64),
+        "yes" if same else "NO")
+    print(line)
+    return line

@@ -162,7 +162,8 @@ def test_read_only_options_and_kernel_options():
     for key, good, bads in ((P.PS_OPT_BULK_TILE, (0, 256, 1024, 8192), (100, 384, 16384, -1)),
                             (P.PS_OPT_BULK_STAGES, (2, 8), (1, 9)),
                             (P.PS_OPT_BULK_WAIT_LIMIT, (16, 1 << 20), (0, 15)),
-                            (P.PS_OPT_BULK_SELFTEST, (0, 1), (2, -1))):
+                            (P.PS_OPT_BULK_SELFTEST, (0, 1), (2, -1)),
+                            (P.PS_OPT_ZIGZAG, (0, 1), (2, -1))):
         for g in good:
             assert P.ps_set_option(h, key, g) == 0
             assert P.ps_get_option(h, key, C.byref(v)) == 0 and v.value == g
@@ -452,3 +453,23 @@ def test_plain_c_client_compiles_links_and_runs(tmp_path):
                     "-L", libdir, "-l:libsoftsync_ps.so", "-Wl,-rpath," + libdir], check=True)
     out = subprocess.run([exe], capture_output=True, text=True)
     assert out.returncode == 0 and "c client ok" in out.stdout, out.stdout + out.stderr
+
+
+@pytest.mark.gpu
+def test_c_latency_client_drives_the_small_configuration_from_c(tmp_path):
+    """The per-update latency figures of the small (launch-bound) configurations come from a C program,
+    tests/c_latency_client.c, so that no interpreter sits between the calls.  Built with gcc against the
+    library and the CUDA runtime, run for a short while; its lines are printed (pytest -s shows them)."""
+    import subprocess
+    libdir = os.path.join(ROOT, "paper_1511_05950_b200")
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    exe = str(tmp_path / "c_latency_client")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-O2", "-I", os.path.join(ROOT, "include"),
+                    "-isystem", os.path.join(cuda, "include"), os.path.join(ROOT, "tests", "c_latency_client.c"),
+                    "-o", exe, "-L", libdir, "-l:libsoftsync_ps.so", "-Wl,-rpath," + libdir,
+                    "-L", os.path.join(cuda, "lib64"), "-lcudart", "-Wl,-rpath," + os.path.join(cuda, "lib64")], check=True)
+    out = subprocess.run([exe, "4000"], capture_output=True, text=True, timeout=300)
+    print(out.stdout)
+    assert out.returncode == 0 and "c latency client ok" in out.stdout, out.stdout + out.stderr
+    per_update = [float(line.split()[-4]) for line in out.stdout.splitlines() if line.endswith("us per update")]
+    assert len(per_update) == 5 and all(0.0 < x < 200.0 for x in per_update)

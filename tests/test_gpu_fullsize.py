@@ -13,7 +13,7 @@ import torch
 
 import paper_1511_05950_b200 as P
 from oracle import reference as R
-from tests.gpu_harness import TORCH_DTYPE, as_reference_grad, assert_logs_equal
+from tests.gpu_harness import TORCH_DTYPE, as_reference_grad, assert_logs_equal, parity_line
 from tests.helpers import PULL, rel_l2
 from workloads import configs, generators as G
 
@@ -96,9 +96,7 @@ def run_full(cfg, lazy, num_pushes=None, overlap=False):
     w64, v64 = refs[64].state()
     tol = 1e-3 if cfg.grad_dtype == "bf16" else 1e-5
     assert rel_l2(w, w64) <= tol and rel_l2(v, v64) <= tol
-    run_full.last_stats = {"gpu_vs_fp64_w": rel_l2(w, w64), "gpu_vs_fp64_v": rel_l2(v, v64),
-                           "fp32ref_vs_fp64_w": rel_l2(w32, w64), "fp32ref_vs_fp64_v": rel_l2(v32, v64),
-                           "sampled_elements": int(idx.numel()), "updates": int(pushes // cfg.c)}
+    parity_line(cfg.name, n, pushes // cfg.c, "%d sampled elements" % idx.numel(), w, v, w32, v32, w64, v64)
     return log
 
 

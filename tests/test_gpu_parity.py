@@ -11,7 +11,7 @@ import torch
 
 import paper_1511_05950_b200 as P
 from oracle import reference as R
-from tests.gpu_harness import run_pair, assert_parity
+from tests.gpu_harness import run_pair, assert_parity, parity_line
 from workloads import configs, generators as G, layouts
 
 pytestmark = pytest.mark.gpu
@@ -30,6 +30,8 @@ def run_config(cfg, num_pushes=None, layout=None, **kw):
                                kinds, learners, w0, cfg.seed, **kw)
     tol = TOL_BF16 if cfg.grad_dtype == "bf16" else TOL_FP32
     worst = assert_parity(w, v, log, refs, tol, layout)
+    parity_line(cfg.name, layout.num_params, pushes // cfg.c, "all elements", w, v, refs[32][0], refs[32][1],
+                refs[64][0], refs[64][1])
     return worst, log
 
 
@@ -106,6 +108,7 @@ def test_temporal_fusion_is_invisible(lam, n, fuse_t, grad_dtype):
     {P.PS_OPT_KERNEL: P.PS_KERNEL_SCALAR}, {P.PS_OPT_KERNEL: P.PS_KERNEL_VECTOR},
     {P.PS_OPT_BLOCK_THREADS: 128}, {P.PS_OPT_BLOCK_THREADS: 256}, {P.PS_OPT_BLOCK_THREADS: 512},
     {P.PS_OPT_KERNEL: P.PS_KERNEL_SCALAR, P.PS_OPT_BLOCK_THREADS: 512},
+    {P.PS_OPT_ZIGZAG: 0}, {P.PS_OPT_ZIGZAG: 0, P.PS_OPT_OVERLAP_LAUNCH: 1},
     {P.PS_OPT_KERNEL: P.PS_KERNEL_BULK},
     {P.PS_OPT_KERNEL: P.PS_KERNEL_BULK, P.PS_OPT_BULK_TILE: 256, P.PS_OPT_BULK_STAGES: 2},
     {P.PS_OPT_KERNEL: P.PS_KERNEL_BULK, P.PS_OPT_BULK_TILE: 512, P.PS_OPT_BULK_STAGES: 8, P.PS_OPT_BLOCK_THREADS: 128},

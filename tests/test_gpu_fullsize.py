@@ -194,6 +194,8 @@ def test_every_element_at_full_size(cfg, updates, layers):
     assert launches == updates // cfg.fuse_t and launches % 2 == 0 and ps.get_option(P.PS_OPT_LAUNCHES_SCALAR) == 0
     ref.assert_state_equals(ps.w.cpu().numpy(), ps.v.cpu().numpy())
     assert_logs_equal(ps.update_log(), ref.parts[0][2].log())
+    print("PARITY | %s%s | %d | %d | all elements, %d launches | theta, v and log bit-equal to the fp32 reference |"
+          % (cfg.name, " + layer multipliers" if layers else "", n, updates, launches))
     ps.destroy()
     ref.close()
 

@@ -506,6 +506,7 @@ def test_contiguous_shards_need_no_synchronisation():
         sh = P.ParameterServer(b - a, lam, n, 0.02, 0.9, 5e-4, fuse_t=2, device=dev, state=(wbuf[a:b], vbuf[a:b]))
         sh.init_weights(w0[a:b].contiguous())
         shards.append((a, b, sh))
+    shards[1][2].bind_staging(2 * (lam // n) * 2)          # the middle shard receives into its own slots
     pulled, counts = {}, {}
     for k, l in zip(kinds.tolist(), learners.tolist()):
         if k == 0:
@@ -516,7 +517,12 @@ def test_contiguous_shards_need_no_synchronisation():
         g = G.gradient(14, l, c_, n_el, 1e-3, device=dev)
         whole.push_gradient(l, g, pulled[l])
         for a, b, sh in shards:
-            sh.push_gradient(l, g[a:b], pulled[l])         # slice a of the same gradient goes to shard a
+            if sh is shards[1][2]:                         # scattered push: the learner writes its slice straight
+                sid, slot = sh.acquire_slot()              # into a receive slot of the shard that owns the range
+                slot.copy_(g[a:b])
+                sh.push_slot(l, sid, pulled[l])
+            else:
+                sh.push_gradient(l, g[a:b], pulled[l])     # slice a of the same gradient goes to shard a
         if whole.timestamps()[1] - whole.timestamps()[0] >= 2:
             whole.apply_update()
             for _, _, sh in shards:

@@ -202,6 +202,8 @@ def build_server(P, cfg, args, dev, rank, fuse_t):
                                  [0.0 if seg.is_bias else 1.0 for seg in layout.segments])
     if args.bf16_mirror:
         ps.bind_weight_mirror()                    # every pass also writes theta as bf16 (2 more bytes per element)
+    if args.replicas:                              # every pass also writes theta into R further fp32 buffers
+        ps.bind_weight_replicas([torch.empty(n, dtype=torch.float32, device=dev) for _ in range(args.replicas)])
     return ps, n
 
 
@@ -356,12 +358,12 @@ def run_ours(args, cfg, rank, world, local_rank):
     else:
         value = whole_job_value(world, elems_per_step, args.steps, median_ms)
         e2e_value = whole_job_value(world, elems_per_step, e2e_steps, e2e_ms) if e2e_steps else None
-    abytes = algorithmic_bytes(n, cfg.c * fuse_t, gbytes) + (2 * n if args.bf16_mirror else 0)
+    abytes = algorithmic_bytes(n, cfg.c * fuse_t, gbytes) + (2 * n if args.bf16_mirror else 0) + 4 * n * args.replicas
     kern_ms = stat["median"]
     achieved = abytes / (kern_ms * 1e-3) / 1e9
     kernel_name = {1: "scalar", 2: "vector", 3: "bulk"}.get(facts["last_kernel"], "none")
     traffic, traffic_from = traffic_for(cfg.name, kernel_name, cfg.grad_dtype, cfg.c, fuse_t, args.block_threads,
-                                        args.bf16_mirror, args.layer_multipliers)
+                                        args.bf16_mirror or args.replicas, args.layer_multipliers)
     if (args.no_overlap or args.no_zigzag) and traffic is not None:
         traffic, traffic_from = None, "the recorded capture used programmatic dependent launches and alternating traversal"
     mid = sorted(reps, key=lambda r: r["ms"])[len(reps) // 2]
@@ -377,6 +379,7 @@ def run_ours(args, cfg, rank, world, local_rank):
             "grad_dtype": cfg.grad_dtype, "arrivals": cfg.arrival_model, "alpha0": cfg.alpha0,
             "momentum": cfg.momentum, "weight_decay": cfg.weight_decay, "modulation": cfg.modulation,
             "bf16_mirror": bool(args.bf16_mirror), "layer_multipliers": bool(args.layer_multipliers),
+            "weight_replicas": args.replicas,
             "kernel": kernel_name, "kernel_launches": facts["launches"],
             "launch": "ordinary" if args.no_overlap else "programmatic dependent launch (PS_OPT_OVERLAP_LAUNCH=1)",
             "traversal": "forward" if args.no_zigzag else "alternating direction from launch to launch",
@@ -668,6 +671,9 @@ def main():
     ap.add_argument("--no-zigzag", action="store_true", help="every launch walks the vector forward (PS_OPT_ZIGZAG=0)")
     ap.add_argument("--bf16-mirror", action="store_true",
                     help="variant: keep a bf16 copy of the weights current in the same pass (+2 bytes per element)")
+    ap.add_argument("--replicas", type=int, default=0, choices=range(0, 9),
+                    help="variant: the update pass also stores theta into this many further fp32 buffers "
+                         "(the fused weight broadcast of a sharded server; here all in this GPU's memory)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for profiler captures)")
     ap.add_argument("--num-params", type=int, default=0,
                     help="run the workload's protocol on a flat vector of this many parameters (profiler captures)")
@@ -717,7 +723,7 @@ def main():
     result, e2e_detail = run_ours(args, cfg, rank, world, local_rank)
     default_run = (args.workload == "large_softsync" and not args.num_params and not args.total_params
                    and args.kernel == "auto" and not args.bf16_mirror and not args.layer_multipliers
-                   and not args.no_zigzag)
+                   and not args.no_zigzag and not args.replicas)
     if default_run and not args.no_second_config:
         result["configs"] = {"large_stale_bf16": second_config(args, rank, world, local_rank)}
     if rank == 0:

@@ -128,6 +128,7 @@ enum ps_kernel_choice {
 #define PS_MAX_FUSE_T 16                  /* largest temporal-fusion depth */
 #define PS_MAX_ENTRIES 512                /* largest T * c one kernel pass takes; T is clamped to fit */
 #define PS_MAX_LAYERS 64                  /* largest layer table of ps_set_layer_multipliers */
+#define PS_MAX_REPLICAS 8                 /* most weight replicas of ps_bind_weight_replicas */
 
 /* One gradient's part in one weight update; what the server decided, for checking
  * against Section 2.1 (timestamp, staleness) and Eq. 2-3 (grouping, scale). */
@@ -174,6 +175,20 @@ int ps_init_weights(ps_t *ps, const float *w_src, int src_is_host);
  * read it in place after the update, or take a copy with ps_pull_weights_bf16.  NULL unbinds.
  * Not in the paper (its weights are 4-byte, Section 4.1). */
 int ps_bind_weight_mirror(ps_t *ps, void *mirror_bf16_dev);
+
+/* Weight broadcast fused into the update.  Section 2.2 has the server send the updated weights to the learners;
+ * Section 2.3 shards the server.  Binds up to PS_MAX_REPLICAS further fp32 buffers of num_params elements that
+ * from now on always hold theta as well: they are filled at once (and by ps_init_weights), and every
+ * ps_apply_update stores the new theta there in the same pass that computes it (4 more bytes written per element
+ * and replica, nothing more read).  A replica may be memory of ANOTHER GPU that this GPU can address (a peer
+ * mapping; the caller obtains it): the kernel only ever stores to a replica, so the data crosses NVLink once, as
+ * remote writes, while the update runs.  With one shard per GPU and, on every GPU, a full-length buffer into
+ * whose range [lo_g, hi_g) shard g writes, a learner's weight pull is a read of its own GPU's buffer: the
+ * all-gather has already happened, tile by tile, inside the update kernels.  The caller orders a learner's read
+ * after the update (ps_synchronize on the owning servers, then its own cross-GPU barrier).
+ * replicas_dev: HOST array of `count` device pointers, copied; 4-byte aligned (16 keeps the vector kernel);
+ * must not overlap theta or v.  count = 0 unbinds.  Only while no complete group is pending. */
+int ps_bind_weight_replicas(ps_t *ps, int count, float *const *replicas_dev);
 
 /* Binds `num_slots` caller-owned device slots of `slot_bytes` each (a multiple of 16, at least
  * num_params * gradient size; base 16-byte aligned) that ps_push_gradient_host copies into. */

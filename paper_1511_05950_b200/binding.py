@@ -32,7 +32,7 @@ PS_GRAD_FP32, PS_GRAD_BF16 = 0, 1
  PS_OPT_BULK_TILE, PS_OPT_BULK_STAGES, PS_OPT_BULK_WAIT_LIMIT, PS_OPT_BULK_SELFTEST, PS_OPT_ZIGZAG) = range(1, 21)
 PS_PROTOCOL_SOFTSYNC, PS_PROTOCOL_HARDSYNC = 0, 1
 PS_KERNEL_AUTO, PS_KERNEL_SCALAR, PS_KERNEL_VECTOR, PS_KERNEL_BULK = 0, 1, 2, 3
-PS_MAX_GROUP, PS_MAX_FUSE_T, PS_MAX_ENTRIES, PS_MAX_LAYERS = 256, 16, 512, 64
+PS_MAX_GROUP, PS_MAX_FUSE_T, PS_MAX_ENTRIES, PS_MAX_LAYERS, PS_MAX_REPLICAS = 256, 16, 512, 64, 8
 
 MODULATIONS = {"constant": PS_MOD_CONSTANT, "inv_staleness": PS_MOD_INV_STALENESS, "exp_staleness": PS_MOD_EXP_STALENESS}
 KERNELS = {"auto": PS_KERNEL_AUTO, "scalar": PS_KERNEL_SCALAR, "vector": PS_KERNEL_VECTOR, "bulk": PS_KERNEL_BULK}
@@ -51,7 +51,7 @@ EXPORTS = (
     "ps_slot_wait", "ps_slot_written", "ps_kernel_status", "ps_pull_weights", "ps_pull_weights_host", "ps_pull_weights_host_async",
     "ps_push_gradient", "ps_push_gradient_host", "ps_acquire_slot", "ps_push_slot", "ps_release_slot", "ps_apply_update", "ps_flush", "ps_synchronize",
     "ps_get_update_log", "ps_peek_state", "ps_export_state", "ps_import_state", "ps_kernel_time", "ps_last_cuda_error", "ps_status_string",
-    "ps_fused_update_static",
+    "ps_fused_update_static", "ps_bind_weight_replicas",
 )
 
 
@@ -76,6 +76,7 @@ def _load() -> C.CDLL:
         "ps_init_weights": [vp, vp, i32],
         "ps_bind_staging": [vp, vp, i64, i32],
         "ps_bind_weight_mirror": [vp, vp],
+        "ps_bind_weight_replicas": [vp, i32, C.POINTER(vp)],
         "ps_pull_weights_bf16": [vp, vp, C.POINTER(i64)],
         "ps_set_option": [vp, i32, i64],
         "ps_get_option": [vp, i32, C.POINTER(i64)],
@@ -122,6 +123,7 @@ ps_bind_state = lib.ps_bind_state
 ps_init_weights = lib.ps_init_weights
 ps_bind_staging = lib.ps_bind_staging
 ps_bind_weight_mirror = lib.ps_bind_weight_mirror
+ps_bind_weight_replicas = lib.ps_bind_weight_replicas
 ps_pull_weights_bf16 = lib.ps_pull_weights_bf16
 ps_set_option = lib.ps_set_option
 ps_get_option = lib.ps_get_option
@@ -235,6 +237,7 @@ class ParameterServer:
         self._host_held = []          # pinned host gradients whose upload may still be in flight
         self._staging = None
         self.w = self.v = self.mirror = None
+        self.replicas = []
         if device is None and (allocate or state is not None) and num_params > 0:
             device = torch.device("cuda", torch.cuda.current_device())
         self.device = device
@@ -301,6 +304,16 @@ class ParameterServer:
         _check(ps_bind_weight_mirror(self._h, mirror.data_ptr()), "ps_bind_weight_mirror")
         self.mirror = mirror
         return mirror
+
+    def bind_weight_replicas(self, replicas) -> None:
+        """Keep further fp32 copies of the weights current: every update stores the new theta into each tensor of
+        `replicas` as well (tensors of num_params fp32 this GPU can address; an empty list unbinds)."""
+        replicas = list(replicas)
+        for t in replicas:
+            require_tensor(t, torch.float32, self.num_params, "weight replica", on_gpu=True)
+        ptrs = (C.c_void_p * max(1, len(replicas)))(*[t.data_ptr() for t in replicas])
+        _check(ps_bind_weight_replicas(self._h, len(replicas), ptrs), "ps_bind_weight_replicas")
+        self.replicas = replicas
 
     def set_option(self, key: int, value: int) -> None:
         _check(ps_set_option(self._h, key, int(value)), "ps_set_option")

@@ -50,6 +50,8 @@ struct ps_ctx {
 
     float *w = nullptr, *v = nullptr;
     unsigned short *mirror = nullptr;      // optional caller-owned bf16 copy of theta
+    int num_replicas = 0;                  // optional caller-owned fp32 copies of theta (ps_bind_weight_replicas)
+    float *replicas[PS_MAX_REPLICAS] = {};
     char *staging = nullptr;
     int64_t slot_bytes = 0;
     std::vector<int> free_slots;
@@ -305,6 +307,8 @@ void build_launch(ps_ctx *ps, int T, Params<MAXE, LAYERS> &p, std::vector<ps_log
     p.overlap = ps->overlap_launch;
     p.reverse = ps->zigzag ? static_cast<int>(ps->launches & 1) : 0;   // zig-zag over the vector from launch to launch
     p.mirror = ps->mirror;
+    p.nrep = ps->num_replicas;
+    for (int r = 0; r < ps->num_replicas; ++r) p.rep[r] = ps->replicas[r];
     p.layers.count = 0;
     if constexpr (LAYERS) {
         p.layers.count = ps->num_layers;
@@ -316,7 +320,8 @@ void build_launch(ps_ctx *ps, int T, Params<MAXE, LAYERS> &p, std::vector<ps_log
     // bf16 mirror in 8-byte pieces.  The bulk copies need 16 bytes everywhere.
     const uintptr_t grad_align = ps->grad_dtype == PS_GRAD_BF16 ? 8 : 16;
     vector_ok = aligned16(ps->w) && aligned16(ps->v) && aligned_to(ps->mirror, 8);
-    bulk_ok = aligned16(ps->w) && aligned16(ps->v) && aligned_to(ps->mirror, 8);
+    for (int r = 0; r < ps->num_replicas; ++r) vector_ok = vector_ok && aligned16(ps->replicas[r]);
+    bulk_ok = vector_ok;
     const double wd = static_cast<double>(ps->weight_decay);
     for (int t = 0; t < T; ++t) {
         std::vector<Entry> &grp = ps->ready[t];
@@ -362,10 +367,14 @@ int order_after_readback(ps_ctx *ps)
     return PS_OK;
 }
 
-// Rewrites the whole bf16 mirror from theta (set-up paths; updates keep it current themselves).
+// Rewrites the bf16 mirror and the fp32 replicas from theta (set-up paths; updates keep them current themselves).
 int refresh_mirror(ps_ctx *ps)
 {
-    if (!ps->mirror || !ps->w || ps->n == 0) return PS_OK;
+    if (!ps->w || ps->n == 0) return PS_OK;
+    for (int r = 0; r < ps->num_replicas; ++r)
+        PS_CUDA(ps, cudaMemcpyAsync(ps->replicas[r], ps->w, static_cast<size_t>(ps->n) * sizeof(float),
+                                    cudaMemcpyDefault, ps->stream));
+    if (!ps->mirror) return PS_OK;
     const int threads = 256;
     const long long want = (ps->n + threads - 1) / threads;
     const int blocks = static_cast<int>(std::min<long long>(want, static_cast<long long>(ps->sm_count) * 32));
@@ -625,6 +634,27 @@ int ps_bind_weight_mirror(ps_t *ps, void *mirror_dev)
         if (mirror_dev && (mirror_dev == ps->w || mirror_dev == ps->v)) return PS_ERR_INVALID_ARG;
         if (!ps->ready.empty()) return PS_ERR_INVALID_ARG;               // apply or flush first
         ps->mirror = static_cast<unsigned short *>(mirror_dev);
+        return refresh_mirror(ps);
+    } PS_CATCH_ALL
+}
+
+int ps_bind_weight_replicas(ps_t *ps, int count, float *const *replicas_dev)
+{
+    try {
+        if (!is_live(ps) || count < 0 || count > PS_MAX_REPLICAS || (count > 0 && !replicas_dev)) return PS_ERR_INVALID_ARG;
+        if (!ps->ready.empty()) return PS_ERR_INVALID_ARG;               // apply or flush first
+        const uintptr_t bytes = static_cast<uintptr_t>(ps->n) * sizeof(float);
+        for (int r = 0; r < count; ++r) {
+            const uintptr_t a = reinterpret_cast<uintptr_t>(replicas_dev[r]);
+            if (!a || (a & 3u)) return PS_ERR_INVALID_ARG;
+            for (const void *other : {static_cast<const void *>(ps->w), static_cast<const void *>(ps->v)}) {
+                const uintptr_t b = reinterpret_cast<uintptr_t>(other);
+                if (b && (a < b ? b - a : a - b) < bytes) return PS_ERR_INVALID_ARG;     // overlaps theta or v
+            }
+        }
+        DeviceGuard on_device(ps);
+        ps->num_replicas = count;
+        for (int r = 0; r < count; ++r) ps->replicas[r] = replicas_dev[r];
         return refresh_mirror(ps);
     } PS_CATCH_ALL
 }
@@ -1206,7 +1236,7 @@ extern "C" int ps_fused_update_static(float *w_dev, float *v_dev, int64_t num_pa
     StaticParams p;
     p.w = w_dev; p.v = v_dev; p.n = num_params;
     p.momentum = momentum; p.T = 1; p.c = c;
-    p.overlap = 0; p.reverse = 0; p.mirror = nullptr;
+    p.overlap = 0; p.reverse = 0; p.mirror = nullptr; p.nrep = 0;
     p.layers.count = 0;
     p.d[0] = decay;
     for (int l = 0; l < c; ++l) { p.s[l] = scales_host[l]; p.g[l] = grads_dev[l]; }

@@ -22,6 +22,7 @@
 namespace softsync {
 
 constexpr int kMaxFuseT = 16;
+constexpr int kMaxReplicas = 8;
 
 // Per-layer learning-rate / decay multipliers: layer q ends before element end[q].
 template <int MAXSEG>
@@ -46,6 +47,8 @@ struct LaunchParams {
     int overlap;          // 1: launched as a programmatic dependent; gradients may be fetched early
     int reverse;          // 1: blocks walk the vector from its end (alternates from launch to launch)
     unsigned short *mirror;   // optional bf16 copy of theta, rewritten by every pass (nullptr: none)
+    int nrep;                 // further fp32 copies of this range of theta, written by the same pass: the weight
+    float *rep[kMaxReplicas]; // broadcast of a sharded server (a destination may be another GPU's memory)
     float d[kMaxFuseT];
     float s[MAXE];
     const void *g[MAXE];
@@ -120,6 +123,22 @@ __device__ __forceinline__ void store_state(float *p, const float (&x)[VEC])
 #pragma unroll
         for (int j = 0; j < VEC / 4; ++j)
             __stcs(reinterpret_cast<float4 *>(p) + j, make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]));
+    }
+}
+
+// theta into its replicas.  Plain stores: a replica may live in a peer GPU's memory, where they travel as
+// ordinary remote writes over NVLink (no load ever touches a replica).
+template <int VEC, typename Params>
+__device__ __forceinline__ void store_replicas(const Params &p, long long first, const float (&x)[VEC])
+{
+    for (int r = 0; r < p.nrep; ++r) {
+        float *dst = p.rep[r] + first;
+        if constexpr (VEC == 1) {
+            *dst = x[0];
+        } else {
+            static_assert(VEC == 4, "fragments hold one or four elements");
+            *reinterpret_cast<float4 *>(dst) = make_float4(x[0], x[1], x[2], x[3]);
+        }
     }
 }
 
@@ -296,6 +315,7 @@ __device__ __forceinline__ void update_fragment(const Params &p, long long i, lo
     store_state<VEC>(p.w + first, f.w);
     store_state<VEC>(p.v + first, f.v);
     if (p.mirror) store_mirror<VEC>(p.mirror + first, f.w);
+    if (p.nrep) store_replicas<VEC>(p, first, f.w);
 }
 
 // One element, any number of entries, with the layer looked up for that element.
@@ -445,6 +465,7 @@ __device__ __forceinline__ void update_from_stage(const Params &p, const unsigne
     store_state<VEC>(p.w + first, f.w);
     store_state<VEC>(p.v + first, f.v);
     if (p.mirror) store_mirror<VEC>(p.mirror + first, f.w);
+    if (p.nrep) store_replicas<VEC>(p, first, f.w);
 }
 
 // BLOCK_RECORDS: plan.status is an array with one record per block of the grid (each block that gives up

@@ -5,7 +5,9 @@ The paper shards its parameter server and notes that the shards need no synchron
 range.  Here rank r of a torch.distributed group owns elements [bounds[r], bounds[r+1]) and runs an ordinary
 server (the C-ABI library) on them.  Every rank must see the same sequence of pulls and pushes; a push hands
 each rank its own slice of the gradient; the only exchange is the all-gather that assembles the full weight
-vector for a pull.  With a world size of one this is the plain server.
+vector for a pull, or, with replica buffers bound, the stores with which every shard's update kernel writes its
+range of the new weights into every GPU's buffer while it computes them.  With a world size of one this is the
+plain server.
 """
 from __future__ import annotations
 
@@ -53,6 +55,7 @@ class ShardedParameterServer:
         self.local = server_factory(self.hi - self.lo, num_learners, n, alpha0, momentum, weight_decay,
                                     modulation, grad_dtype, fuse_t, device=device)
         self._max_shard = max(b - a for a, b in zip(self.bounds[:-1], self.bounds[1:]))
+        self.replica_buffers = []
 
     # -- set-up ---------------------------------------------------------------
     def init_weights(self, w0_full: torch.Tensor) -> None:
@@ -90,6 +93,31 @@ class ShardedParameterServer:
         if grad_slice.numel() != self.hi - self.lo:
             raise ValueError("slice of %d elements for a shard of %d" % (grad_slice.numel(), self.hi - self.lo))
         return self.local.push_gradient(learner, grad_slice, ts)
+
+    # -- weight broadcast fused into the update ----------------------------------
+    def bind_replica_buffers(self, full_buffers) -> None:
+        """`full_buffers`: full-length fp32 tensors that THIS GPU can address, one per GPU whose learners should
+        find the whole weight vector in their own memory (this GPU's own buffer, and peer mappings of the
+        other GPUs' buffers, which the caller sets up).  This rank's update kernel then stores its range of the
+        new theta into every one of them while it computes it: after all ranks' updates the buffers hold the
+        assembled weights and a pull is a local read (`pull_weights_from_replica`).  The kernel only stores to
+        the buffers; nothing of this library ever loads from another GPU's memory."""
+        for t in full_buffers:
+            if t.numel() != self.num_params or t.dtype != torch.float32:
+                raise ValueError("a replica buffer holds the whole fp32 weight vector")
+        self.replica_buffers = list(full_buffers)
+        self.local.bind_weight_replicas([t[self.lo:self.hi] for t in self.replica_buffers])
+
+    def pull_weights_from_replica(self) -> int:
+        """The pull when replica buffers are bound: every rank waits for its own updates, the ranks meet at a
+        barrier (control only, no weight bytes move), and this GPU's own replica buffer then holds the weights
+        of the returned timestamp."""
+        self.local.flush()
+        ts = self.local.pull_weights()
+        self.local.synchronize()
+        if self.world > 1:
+            dist.barrier(group=self.group)
+        return ts
 
     # receive slots of this rank's shard: a learner on the same GPU writes its slice straight into server memory
     def bind_staging(self, num_slots: int) -> None:

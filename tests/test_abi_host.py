@@ -320,6 +320,26 @@ def test_weight_mirror_argument_checks():
     P.ps_destroy(h)
 
 
+def test_weight_replica_argument_checks():
+    rc, h = make(2, 1)
+    ptrs = (C.c_void_p * 9)(*[0x1000 * (k + 1) for k in range(9)])
+    assert P.ps_bind_weight_replicas(h, 9, ptrs) == P.PS_ERR_INVALID_ARG         # more than PS_MAX_REPLICAS
+    assert P.ps_bind_weight_replicas(h, -1, ptrs) == P.PS_ERR_INVALID_ARG
+    assert P.ps_bind_weight_replicas(h, 2, None) == P.PS_ERR_INVALID_ARG
+    assert P.ps_bind_weight_replicas(None, 1, ptrs) == P.PS_ERR_INVALID_ARG
+    odd = (C.c_void_p * 1)(0x1002)
+    assert P.ps_bind_weight_replicas(h, 1, odd) == P.PS_ERR_INVALID_ARG          # not 4-byte aligned
+    null = (C.c_void_p * 2)(0x1000, None)
+    assert P.ps_bind_weight_replicas(h, 2, null) == P.PS_ERR_INVALID_ARG
+    assert P.ps_bind_weight_replicas(h, 8, ptrs) == 0                            # zero parameters: nothing is written
+    assert P.ps_push_gradient(h, 0, FAKE_GRAD, 0) == P.PS_OK
+    assert P.ps_push_gradient(h, 1, FAKE_GRAD, 0) == P.PS_READY
+    assert P.ps_bind_weight_replicas(h, 0, None) == P.PS_ERR_INVALID_ARG         # a complete group is pending
+    assert P.ps_apply_update(h) == 1
+    assert P.ps_bind_weight_replicas(h, 0, None) == 0                            # unbind
+    P.ps_destroy(h)
+
+
 def test_checkpoint_on_a_group_boundary_resumes_the_same_schedule():
     lam, n, pushes = 6, 2, 120
     c = lam // n

@@ -478,6 +478,110 @@ def test_bf16_weight_mirror_tracks_the_weights(grad_dtype, fuse_t, n_el, misalig
     ps.destroy()
 
 
+@pytest.mark.parametrize("grad_dtype,fuse_t,kernel,misalign", [
+    ("fp32", 1, "auto", 0), ("bf16", 8, "auto", 0), ("fp32", 2, "auto", 1), ("fp32", 1, "bulk", 0), ("bf16", 4, "scalar", 0)])
+def test_weight_replicas_are_written_by_the_update_pass(grad_dtype, fuse_t, kernel, misalign):
+    """ps_bind_weight_replicas: three further fp32 buffers hold theta after set-up and after every update,
+    bit for bit the reference's weights; nothing outside them is touched; a misaligned replica takes the
+    scalar kernel; unbinding stops the writes."""
+    from tests.gpu_harness import as_reference_grad
+    dev = torch.device("cuda", 0)
+    tdt = torch.bfloat16 if grad_dtype == "bf16" else torch.float32
+    lam, n, n_el = 8, 8, 9 * 4096 + 77
+    kinds, learners = R.simulate_arrivals("exp", lam, 48, 23)
+    w0 = G.initial_weights(layouts.flat(n_el), 23)
+    ref = R.ReferencePS(n_el, lam, n, 0.05, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    ps = P.ParameterServer(n_el, lam, n, 0.05, 0.9, 5e-4, grad_dtype=grad_dtype, fuse_t=fuse_t, device=dev)
+    ps.set_option(P.PS_OPT_KERNEL, P.binding.KERNELS[kernel])
+    ps.init_weights(w0.to(dev))
+    guards = [torch.full((n_el + 72,), 7.0, device=dev) for _ in range(3)]
+    offs = [8, 8 + misalign, 8]
+    reps = [gd[o:o + n_el] for gd, o in zip(guards, offs)]
+    ps.bind_weight_replicas(reps)
+    want = lambda: ref.state()[0].astype(np.float32)
+    for r in reps:
+        assert np.array_equal(r.cpu().numpy(), want())                       # filled when bound
+    pulled, counts, ready = {}, {}, 0
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == 0:
+            pulled[l] = ps.pull_weights(); ref.pull(l)
+            continue
+        b = counts.get(l, 0); counts[l] = b + 1
+        g = G.gradient(23, l, b, n_el, 1e-2, dtype=tdt, device=dev)
+        ref.push(l, as_reference_grad(g))
+        ready += ps.push_gradient(l, g, pulled[l])
+        if ready >= fuse_t:
+            ready -= ps.apply_update()
+            if ready == 0:
+                for r in reps:
+                    assert np.array_equal(r.cpu().numpy(), want())
+    ps.flush(); ps.synchronize()
+    assert ps.get_option(P.PS_OPT_LAST_KERNEL) == (P.PS_KERNEL_SCALAR if misalign or kernel == "scalar" else
+                                                   P.binding.KERNELS[kernel] or P.PS_KERNEL_VECTOR)
+    assert np.array_equal(ps.w.cpu().numpy(), want())
+    for gd, o, r in zip(guards, offs, reps):
+        assert np.array_equal(r.cpu().numpy(), want())
+        assert (gd[:o] == 7.0).all() and (gd[o + n_el:] == 7.0).all()
+    ps.bind_weight_replicas([])                                              # unbound: later updates leave them alone
+    before = reps[0].clone()
+    ts = ps.pull_weights()
+    for l in range(lam):
+        ps.push_gradient(l, G.gradient(23, l, 99, n_el, 1e-2, dtype=tdt, device=dev), ts)
+    ps.flush(); ps.synchronize()
+    assert torch.equal(reps[0], before) and not torch.equal(ps.w, before)
+    ps.destroy()
+
+
+def test_shards_assemble_the_weights_in_every_replica_buffer():
+    """The all-gather of the sharded server, fused into the update: three shards over contiguous ranges, and two
+    full-length buffers standing for two GPUs' copies of the weights.  Every shard's update kernel stores its
+    range into both; after the updates both buffers hold the reference's whole weight vector, without any copy
+    or gather at pull time."""
+    from paper_1511_05950_b200.sharded import shard_bounds
+    from tests.gpu_harness import as_reference_grad
+    from tests.helpers import replay_reference
+    dev = torch.device("cuda", 0)
+    n_el, lam, n, world = 100003, 6, 2, 3
+    bounds = shard_bounds(n_el, world)
+    kinds, learners = R.simulate_arrivals("lognormal", lam, 60, 31)
+    w0 = G.initial_weights(layouts.flat(n_el), 31).to(dev)
+    buffers = [torch.zeros(n_el, device=dev) for _ in range(2)]
+    shards = []
+    for a, b in zip(bounds[:-1], bounds[1:]):
+        sh = P.ParameterServer(b - a, lam, n, 0.02, 0.9, 5e-4, fuse_t=2, device=dev)
+        sh.init_weights(w0[a:b].contiguous())
+        sh.bind_weight_replicas([buf[a:b] for buf in buffers])
+        shards.append((a, b, sh))
+    assert all(torch.equal(buf, w0) for buf in buffers)
+    ref = R.ReferencePS(n_el, lam, n, 0.02, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.cpu().numpy())
+    pulled, counts = {}, {}
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == 0:
+            pulled[l] = shards[0][2].pull_weights()
+            assert all(sh.pull_weights() == pulled[l] for _, _, sh in shards) and ref.pull(l) == pulled[l]
+            continue
+        c_ = counts.get(l, 0); counts[l] = c_ + 1
+        g = G.gradient(31, l, c_, n_el, 1e-3, device=dev)
+        ref.push(l, as_reference_grad(g))
+        for a, b, sh in shards:
+            if sh.push_gradient(l, g[a:b], pulled[l]):
+                sh.apply_update()
+        if ref.timestamp % 5 == 0:
+            torch.cuda.synchronize()
+            if all(sh.timestamps()[0] == ref.timestamp for _, _, sh in shards):
+                for buf in buffers:
+                    assert np.array_equal(buf.cpu().numpy(), ref.state()[0].astype(np.float32))
+    for _, _, sh in shards:
+        sh.flush()
+    torch.cuda.synchronize()
+    for buf in buffers:
+        assert np.array_equal(buf.cpu().numpy(), ref.state()[0].astype(np.float32))
+    for _, _, sh in shards:
+        sh.destroy()
+
+
 def test_bf16_pull_needs_a_mirror():
     dev = torch.device("cuda", 0)
     ps = P.ParameterServer(64, 1, 1, 0.1, device=dev)

@@ -187,7 +187,7 @@ int ps_bind_weight_mirror(ps_t *ps, void *mirror_bf16_dev);
  * all-gather has already happened, tile by tile, inside the update kernels.  The caller orders a learner's read
  * after the update (ps_synchronize on the owning servers, then its own cross-GPU barrier).
  * replicas_dev: HOST array of `count` device pointers, copied; 4-byte aligned (16 keeps the vector kernel);
- * must not overlap theta or v.  count = 0 unbinds.  Only while no complete group is pending. */
+ * must not overlap theta, v, the bf16 mirror or one another.  count = 0 unbinds.  Only while no complete group is pending. */
 int ps_bind_weight_replicas(ps_t *ps, int count, float *const *replicas_dev);
 
 /* Binds `num_slots` caller-owned device slots of `slot_bytes` each (a multiple of 16, at least

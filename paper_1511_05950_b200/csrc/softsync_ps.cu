@@ -589,9 +589,17 @@ int ps_bind_state(ps_t *ps, float *w_dev, float *v_dev)
         if (!ps->ready.empty() || !ps->filling.empty()) return PS_ERR_INVALID_ARG;
         if (w_dev == reinterpret_cast<float *>(ps->mirror) || v_dev == reinterpret_cast<float *>(ps->mirror))
             return PS_ERR_INVALID_ARG;
+        for (int r = 0; r < ps->num_replicas; ++r) {                                   // nor a replica bound earlier
+            const uintptr_t bytes = static_cast<uintptr_t>(ps->n) * sizeof(float);
+            const uintptr_t q = reinterpret_cast<uintptr_t>(ps->replicas[r]);
+            for (const float *mine : {w_dev, v_dev}) {
+                const uintptr_t a = reinterpret_cast<uintptr_t>(mine);
+                if ((a < q ? q - a : a - q) < bytes) return PS_ERR_INVALID_ARG;
+            }
+        }
         ps->w = w_dev; ps->v = v_dev;
         DeviceGuard on_device(ps);
-        return refresh_mirror(ps);                        // a mirror bound earlier follows the new theta
+        return refresh_mirror(ps);                        // a mirror and replicas bound earlier follow the new theta
     } PS_CATCH_ALL
 }
 
@@ -651,6 +659,12 @@ int ps_bind_weight_replicas(ps_t *ps, int count, float *const *replicas_dev)
                 const uintptr_t b = reinterpret_cast<uintptr_t>(other);
                 if (b && (a < b ? b - a : a - b) < bytes) return PS_ERR_INVALID_ARG;     // overlaps theta or v
             }
+            for (int q = 0; q < r; ++q) {                                                // or another replica
+                const uintptr_t b = reinterpret_cast<uintptr_t>(replicas_dev[q]);
+                if ((a < b ? b - a : a - b) < bytes) return PS_ERR_INVALID_ARG;
+            }
+            if (const uintptr_t m = reinterpret_cast<uintptr_t>(ps->mirror))             // or the bf16 mirror
+                if (a < m ? m - a < bytes : a - m < bytes / 2) return PS_ERR_INVALID_ARG;
         }
         DeviceGuard on_device(ps);
         ps->num_replicas = count;

@@ -523,6 +523,11 @@ def test_weight_replicas_are_written_by_the_update_pass(grad_dtype, fuse_t, kern
     for gd, o, r in zip(guards, offs, reps):
         assert np.array_equal(r.cpu().numpy(), want())
         assert (gd[:o] == 7.0).all() and (gd[o + n_el:] == 7.0).all()
+    big = torch.zeros(2 * n_el + 8, device=dev)
+    for bad in ([big[:n_el], big[4:4 + n_el]], [big[:n_el], big[:n_el]], [ps.w], [big[:n_el], ps.v]):
+        with pytest.raises(P.SoftsyncError) as e:                            # overlapping one another, theta or v
+            ps.bind_weight_replicas(bad)
+        assert e.value.status == P.PS_ERR_INVALID_ARG
     ps.bind_weight_replicas([])                                              # unbound: later updates leave them alone
     before = reps[0].clone()
     ts = ps.pull_weights()

@@ -12,6 +12,7 @@ import torch
 import paper_1511_05950_b200 as P
 from oracle import reference as R
 from tests.gpu_harness import run_pair, assert_parity, parity_line
+from tests.helpers import PULL
 from workloads import configs, generators as G, layouts
 
 pytestmark = pytest.mark.gpu
@@ -223,6 +224,34 @@ def test_exponential_penalty_matches_reference(rho, grad_dtype, fuse_t):
     assert_parity(w, v, log, refs, TOL_BF16 if grad_dtype == "bf16" else TOL_FP32)
     assert log["tau"].max() >= 5 and np.array_equal(log["sigma"], log["tau"])
     assert len(np.unique(log["scale"])) >= 5
+
+
+@pytest.mark.parametrize("grad_dtype,options,misalign", [
+    ("fp32", None, 0), ("bf16", None, 0), ("fp32", None, 1), ("fp32", {P.PS_OPT_KERNEL: P.PS_KERNEL_BULK}, 0)])
+def test_vanishing_scales_keep_their_denormals(grad_dtype, options, misalign):
+    """The degenerate end of the exponential penalty: a learner that never pulls again pushes gradients whose
+    staleness runs from 118 to 152, so that 0.5^tau passes through the smallest normal fp32 numbers, the
+    denormals and zero.  With momentum 0, decay 0 and theta_0 = 0 the state is made of nothing but those
+    products, and the momentum right after such an update is the bare product s*g: it must not be flushed to
+    zero on the GPU (packed and scalar multiplies alike).  The state is compared after every single update."""
+    from tests.helpers import PUSH
+    lam, n_el = 2, 8197
+    kinds, learners = [PULL, PULL], [0, 1]
+    for u in range(153):
+        if u >= 118 and u % 2 == 0:                     # the stale learner: timestamp 0 for ever
+            kinds.append(PUSH); learners.append(1)
+        kinds += [PUSH, PULL]; learners += [0, 0]
+    kinds, learners = np.asarray(kinds, dtype=np.int32), np.asarray(learners, dtype=np.int32)
+    w0 = torch.zeros(n_el)
+    w, v, log, refs = run_pair(n_el, lam, lam, 1.0, 0.0, 0.0, "exp_staleness", grad_dtype, 1.0, kinds, learners, w0, 97,
+                               penalty_base=0.5, options=options, misalign=misalign, precisions=(32,),
+                               checkpoints=1000)      # v after EVERY update: the stale ones leave it denormal
+    assert_parity(w, v, log, refs, TOL_FP32)
+    stale = log[log["learner"] == 1]
+    tiny = np.finfo(np.float32).tiny
+    assert stale["tau"].min() >= 118 and stale["tau"].max() >= 150
+    assert ((stale["scale"] > 0) & (stale["scale"] < tiny)).any() and (stale["scale"] == 0).any()    # denormal and zero scales
+    assert (stale["scale"] >= tiny).any()
 
 
 def caffe_style_multipliers(layout):

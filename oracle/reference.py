@@ -135,7 +135,10 @@ class ReferencePS:
             self._h = None
 
     def __del__(self):
-        self.close()
+        try:
+            self.close()
+        except Exception:              # interpreter shutdown: the module's globals may be gone already
+            pass
 
     def set_weights(self, w0: np.ndarray) -> None:
         w0 = np.ascontiguousarray(w0, dtype=np.float32)

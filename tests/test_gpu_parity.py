@@ -254,6 +254,52 @@ def test_vanishing_scales_keep_their_denormals(grad_dtype, options, misalign):
     assert (stale["scale"] >= tiny).any()
 
 
+@pytest.mark.parametrize("grad_dtype,fuse_t,kernel", [("fp32", 1, "auto"), ("bf16", 2, "auto"), ("fp32", 2, "scalar"),
+                                                     ("fp32", 1, "bulk"), ("bf16", 1, "bulk")])
+def test_special_values_propagate_like_the_reference(grad_dtype, fuse_t, kernel):
+    """Infinities, NaNs, signed zeros, denormals and the largest finite values in gradients and weights: the
+    same elements become NaN or infinite on both sides, every other element agrees bit for bit (signed zeros
+    included: the comparison is on the bit patterns, NaN payloads excepted)."""
+    from tests.gpu_harness import as_reference_grad
+    dev = torch.device("cuda", 0)
+    tdt = torch.bfloat16 if grad_dtype == "bf16" else torch.float32
+    n_el, lam = 4096 + 5, 2
+    specials = torch.tensor([float("inf"), float("-inf"), float("nan"), -0.0, 0.0, 1e-42, -1e-42, 3.0e38, -3.0e38,
+                             1.17549435e-38, 1.0, -1.0])
+    w0 = G.initial_weights(layouts.flat(n_el), 5)
+    w0[100:100 + specials.numel()] = specials
+    w0[n_el - 3:] = torch.tensor([-0.0, 3.0e38, 1e-42])                        # the ragged tail too
+    ps = P.ParameterServer(n_el, lam, 1, 0.5, 0.9, 5e-4, grad_dtype=grad_dtype, fuse_t=fuse_t, device=dev)
+    ps.set_option(P.PS_OPT_KERNEL, P.binding.KERNELS[kernel])
+    ps.init_weights(w0.to(dev))
+    ref = R.ReferencePS(n_el, lam, 1, 0.5, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    ref.set_weights(w0.numpy())
+    pending = 0
+    for u in range(4):
+        ts = ps.pull_weights()
+        for l in range(lam):
+            ref.pull(l)
+            g = G.gradient(5, l, u, n_el, 1e-2, dtype=torch.float32, device=dev)
+            g[(7 + 13 * u) % 64: (7 + 13 * u) % 64 + specials.numel()] = specials.to(dev)     # over ordinary weights
+            g[100 + u: 100 + u + 4] = specials[u: u + 4].to(dev)                           # over special weights
+            g[n_el - 2] = float("inf") if u == 2 else -0.0
+            if u == 3:
+                g[200], g[201] = float("inf"), float("-inf")                                 # still infinite at the end
+            g = g.to(tdt)
+            ref.push(l, as_reference_grad(g))
+            pending += ps.push_gradient(l, g, ts)
+        if pending >= fuse_t:
+            pending -= ps.apply_update()
+    ps.flush(); ps.synchronize()
+    for got, want in zip((ps.w.cpu().numpy(), ps.v.cpu().numpy()), ref.state()):
+        want = want.astype(np.float32)
+        assert np.array_equal(np.isnan(got), np.isnan(want))
+        ok = ~np.isnan(want)
+        assert np.array_equal(got.view(np.uint32)[ok], want.view(np.uint32)[ok])
+        assert np.isnan(want).any() and np.isinf(want[ok]).any()                 # the case did what it is for
+    ps.destroy()
+
+
 def caffe_style_multipliers(layout):
     """Rate x1 / decay x1 for weights, rate x2 / decay x0 for biases (the usual setting of the Caffe models
     that Section 4.1's networks follow)."""

@@ -110,7 +110,7 @@ def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, g
                     assert r.timestamp == applied
                     wr, vr = r.state()
                     if prec == 32:
-                        assert np.array_equal(wc, wr.astype(np.float32)) and np.array_equal(vc, vr.astype(np.float32))
+                        assert same_bits(wc, wr) and same_bits(vc, vr)
                     else:
                         assert rel_l2(wc, wr) <= tol and rel_l2(vc, vr) <= tol
     ps.flush()
@@ -131,6 +131,17 @@ def run_pair(num_params, lam, n, alpha0, momentum, wd, modulation, grad_dtype, g
     return w, v, log, out
 
 
+def same_bits(x, ref) -> bool:
+    """fp32 arrays equal as bit patterns (so +0 and -0 differ); NaNs must sit in the same places, their
+    payloads may differ."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    ref = np.ascontiguousarray(np.asarray(ref).astype(np.float32))
+    if x.shape != ref.shape or not np.array_equal(np.isnan(x), np.isnan(ref)):
+        return False
+    ok = ~np.isnan(ref)
+    return bool(np.array_equal(x.view(np.uint32)[ok], ref.view(np.uint32)[ok]))
+
+
 def assert_logs_equal(log, rlog):
     for f in ("update", "push_index", "ts_grad", "tau", "sigma", "learner", "position"):
         assert np.array_equal(log[f], rlog[f]), f
@@ -143,8 +154,8 @@ def assert_parity(w, v, log, refs, tol, layout=None):
     if 32 in refs:
         w32, v32, log32 = refs[32]
         assert_logs_equal(log, log32)
-        assert np.array_equal(w, w32.astype(np.float32)), "weights differ from the fp32 reference"
-        assert np.array_equal(v, v32.astype(np.float32)), "momentum differs from the fp32 reference"
+        assert same_bits(w, w32), "weights differ from the fp32 reference"
+        assert same_bits(v, v32), "momentum differs from the fp32 reference"
     if 64 in refs:
         w64, v64, log64 = refs[64]
         worst = max(rel_l2(w, w64), rel_l2(v, v64))
@@ -164,7 +175,7 @@ def parity_line(name, elements, updates, compared, w, v, w32, v32, w64, v64):
     """One row of the parity table (printed by the configuration tests; shown with pytest -s): distance of
     the GPU state from the fp64 reference, distance of the fp32 reference from the fp64 one (what keeping the
     state in fp32 costs by itself), and whether GPU and fp32 reference agree bit for bit."""
-    same = bool(np.array_equal(w, np.asarray(w32, np.float32)) and np.array_equal(v, np.asarray(v32, np.float32)))
+    same = same_bits(w, w32) and same_bits(v, v32)
     line = "PARITY | %s | %d | %d | %s | %.2e | %.2e | %.2e | %.2e | %s |" % (
         name, elements, updates, compared, rel_l2(w, w64), rel_l2(v, v64), rel_l2(w32, w64), rel_l2(v32, v64),
         "yes" if same else "NO")

@@ -13,7 +13,7 @@ import torch
 
 import paper_1511_05950_b200 as P
 from oracle import reference as R
-from tests.gpu_harness import TORCH_DTYPE, as_reference_grad, assert_logs_equal, parity_line
+from tests.gpu_harness import TORCH_DTYPE, as_reference_grad, assert_logs_equal, parity_line, same_bits
 from tests.helpers import PULL, rel_l2
 from workloads import configs, generators as G
 
@@ -92,7 +92,7 @@ def run_full(cfg, lazy, num_pushes=None, overlap=False):
 
     w32, v32 = refs[32].state()
     assert_logs_equal(log, refs[32].log())
-    assert np.array_equal(w, w32.astype(np.float32)) and np.array_equal(v, v32.astype(np.float32))
+    assert same_bits(w, w32) and same_bits(v, v32)
     w64, v64 = refs[64].state()
     tol = 1e-3 if cfg.grad_dtype == "bf16" else 1e-5
     assert rel_l2(w, w64) <= tol and rel_l2(v, v64) <= tol
@@ -142,8 +142,8 @@ class PartitionedReference:
     def assert_state_equals(self, w: np.ndarray, v: np.ndarray):
         for a, b, r in self.parts:
             wr, vr = r.state()
-            assert np.array_equal(w[a:b], wr.astype(np.float32)), "weights differ in [%d, %d)" % (a, b)
-            assert np.array_equal(v[a:b], vr.astype(np.float32)), "momentum differs in [%d, %d)" % (a, b)
+            assert same_bits(w[a:b], wr), "weights differ in [%d, %d)" % (a, b)
+            assert same_bits(v[a:b], vr), "momentum differs in [%d, %d)" % (a, b)
 
     def close(self):
         self.pool.shutdown()

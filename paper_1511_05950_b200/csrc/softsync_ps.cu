@@ -303,7 +303,7 @@ void build_launch(ps_ctx *ps, int T, Params<MAXE, LAYERS> &p, std::vector<ps_log
                   bool &vector_ok, bool &bulk_ok)
 {
     p.w = ps->w; p.v = ps->v; p.n = ps->n;
-    p.momentum = ps->momentum; p.T = T; p.c = ps->c;
+    p.momentum = make_float2(ps->momentum, ps->momentum); p.T = T; p.c = ps->c;
     p.overlap = ps->overlap_launch;
     p.reverse = ps->zigzag ? static_cast<int>(ps->launches & 1) : 0;   // zig-zag over the vector from launch to launch
     p.mirror = ps->mirror;
@@ -336,7 +336,7 @@ void build_launch(ps_ctx *ps, int T, Params<MAXE, LAYERS> &p, std::vector<ps_log
             else                                             // Eq. 3 (sigma = 1 for the constant rate)
                 step = static_cast<double>(en.alpha0) / (static_cast<double>(ps->c) * static_cast<double>(en.sigma));
             const float s = static_cast<float>(step);
-            p.s[t * ps->c + l] = s;
+            p.s[t * ps->c + l] = make_float2(s, s);
             p.g[t * ps->c + l] = en.grad;
             vector_ok = vector_ok && aligned_to(en.grad, grad_align);
             bulk_ok = bulk_ok && aligned16(en.grad);
@@ -344,14 +344,14 @@ void build_launch(ps_ctx *ps, int T, Params<MAXE, LAYERS> &p, std::vector<ps_log
             sum += static_cast<double>(s);
         }
         const float d = static_cast<float>(wd * sum);   // every gradient carries + wd * theta
-        p.d[t] = d;
+        p.d[t] = make_float2(d, d);
         for (int l = 0; l < ps->c; ++l) {
             const Entry &en = grp[l];
             ps_log_entry le;
             le.update = ps->ts_applied + t;
             le.push_index = en.push_index; le.ts_grad = en.ts_grad; le.tau = en.tau; le.sigma = en.sigma;
             le.learner = en.learner; le.position = l;
-            le.scale = p.s[t * ps->c + l]; le.decay = d;
+            le.scale = p.s[t * ps->c + l].x; le.decay = d;
             entries.push_back(le);
         }
     }
@@ -1249,11 +1249,11 @@ extern "C" int ps_fused_update_static(float *w_dev, float *v_dev, int64_t num_pa
 
     StaticParams p;
     p.w = w_dev; p.v = v_dev; p.n = num_params;
-    p.momentum = momentum; p.T = 1; p.c = c;
+    p.momentum = make_float2(momentum, momentum); p.T = 1; p.c = c;
     p.overlap = 0; p.reverse = 0; p.mirror = nullptr; p.nrep = 0;
     p.layers.count = 0;
-    p.d[0] = decay;
-    for (int l = 0; l < c; ++l) { p.s[l] = scales_host[l]; p.g[l] = grads_dev[l]; }
+    p.d[0] = make_float2(decay, decay);
+    for (int l = 0; l < c; ++l) { p.s[l] = make_float2(scales_host[l], scales_host[l]); p.g[l] = grads_dev[l]; }
 
     // the launch shape of the PS_KERNEL_BULK default
     const int gb = grad_dtype == PS_GRAD_BF16 ? 2 : 4;

@@ -41,7 +41,8 @@ struct LaunchParams {
     float *w;
     float *v;
     long long n;          // elements
-    float momentum;
+    float2 momentum;      // every coefficient is held twice (.x == .y): a packed multiply takes the pair as ONE
+                          // 64-bit operand straight from parameter space instead of building it with two moves
     int T;                // groups in this pass
     int c;                // gradients per group
     int overlap;          // 1: launched as a programmatic dependent; gradients may be fetched early
@@ -49,8 +50,8 @@ struct LaunchParams {
     unsigned short *mirror;   // optional bf16 copy of theta, rewritten by every pass (nullptr: none)
     int nrep;                 // further fp32 copies of this range of theta, written by the same pass: the weight
     float *rep[kMaxReplicas]; // broadcast of a sharded server (a destination may be another GPU's memory)
-    float d[kMaxFuseT];
-    float s[MAXE];
+    float2 d[kMaxFuseT];
+    float2 s[MAXE];
     const void *g[MAXE];
     LayerTable<MAXSEG> layers;    // used by the LAYERS instantiations only (MAXSEG = 1 otherwise)
 };
@@ -213,7 +214,26 @@ __device__ __forceinline__ void sub_pair(float &x0, float &x1, float a0, float a
     asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(R) : "l"(A), "l"(B));
     asm("mov.b64 {%0,%1}, %2;" : "=f"(x0), "=f"(x1) : "l"(R));
 }
+// the same with the multiplier already a pair (a.x == a.y): a launch parameter
+__device__ __forceinline__ void mul_pair(float &x0, float &x1, const float2 &a, float b0, float b1)
+{
+    unsigned long long A = *reinterpret_cast<const unsigned long long *>(&a), B, R;
+    asm("mov.b64 %0, {%1,%2};" : "=l"(B) : "f"(b0), "f"(b1));
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(R) : "l"(A), "l"(B));
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(x0), "=f"(x1) : "l"(R));
+}
 // x[j] = a * y[j], every product rounded once
+template <int VEC>
+__device__ __forceinline__ void scale(float (&x)[VEC], const float2 &a, const float (&y)[VEC])
+{
+    if constexpr (VEC == 4) {
+        mul_pair(x[0], x[1], a, y[0], y[1]);
+        mul_pair(x[2], x[3], a, y[2], y[3]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) x[j] = __fmul_rn(a.x, y[j]);
+    }
+}
 template <int VEC>
 __device__ __forceinline__ void scale(float (&x)[VEC], float a, const float (&y)[VEC])
 {
@@ -239,11 +259,10 @@ __device__ __forceinline__ void consume(const Params &p, Fragment<VEC> &f, const
     widen(r, g);
     scale<VEC>(prod, p.s[e], g);
     bool complete = true;
-    float d;
+    int t = e;                                           // CT = 1: entry e is group e
     if constexpr (CT == 1) {
 #pragma unroll
         for (int j = 0; j < VEC; ++j) f.acc[j] = prod[j];
-        d = p.d[e];
     } else {
         if (f.l == 0) {
 #pragma unroll
@@ -253,14 +272,13 @@ __device__ __forceinline__ void consume(const Params &p, Fragment<VEC> &f, const
             for (int j = 0; j < VEC; ++j) f.acc[j] = __fadd_rn(f.acc[j], prod[j]);
         }
         complete = ++f.l == p.c;
-        if (complete) { d = p.d[f.t++]; f.l = 0; }
+        if (complete) { t = f.t++; f.l = 0; }
     }
     if (complete) {                                      // group complete: one weight update
-        const float m = p.momentum;
-        if constexpr (LAYERS) d = __fmul_rn(f.dm, d);
         float dw[VEC], mv[VEC], tt[VEC];
-        scale<VEC>(dw, d, f.w);
-        scale<VEC>(mv, m, f.v);
+        if constexpr (LAYERS) scale<VEC>(dw, __fmul_rn(f.dm, p.d[t].x), f.w);
+        else scale<VEC>(dw, p.d[t], f.w);
+        scale<VEC>(mv, p.momentum, f.v);
 #pragma unroll
         for (int j = 0; j < VEC; ++j) tt[j] = __fadd_rn(f.acc[j], dw[j]);
         if constexpr (LAYERS) scale<VEC>(tt, f.lm, tt);

@@ -164,9 +164,9 @@ NOMINAL_HBM_GBS = 8000.0
 # a figure only when it launches that same instantiation in the same way; anything else gets null and why.
 TRAFFIC_CAPTURES = {
     ("large_softsync", "vector", "fp32", 4, 1, 128, False, False):
-        (1.9141e9, "profiles/softsync_update_fp32_c4_large_softsync.md"),
+        (1.9124e9, "profiles/softsync_update_fp32_c4_large_softsync.md"),
     ("large_stale_bf16", "vector", "bf16", 1, 8, 128, False, False):
-        (1.9160e9, "profiles/softsync_update_bf16_c1_T8_large_stale_bf16.md"),
+        (1.9147e9, "profiles/softsync_update_bf16_c1_T8_large_stale_bf16.md"),
 }
 
 

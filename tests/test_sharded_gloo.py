@@ -67,7 +67,18 @@ class ReferenceBackedServer:
 
     def push_gradient(self, learner, grad, ts):
         self.elements_received += grad.numel()
-        return self.ref.push(learner, grad.contiguous().numpy(), timestamp=ts)
+        fired = self.ref.push(learner, grad.contiguous().numpy(), timestamp=ts)
+        if fired:                                 # the update "kernel" also stores theta into every replica
+            self._write_replicas()
+        return fired
+
+    def bind_weight_replicas(self, replicas):
+        self.replicas = list(replicas)
+        self._write_replicas()
+
+    def _write_replicas(self):
+        for r in getattr(self, "replicas", []):
+            r.copy_(torch.from_numpy(self.ref.state()[0].astype(np.float32)))
 
     def apply_update(self):
         return 1
@@ -206,20 +217,61 @@ def _worker_library_state_machine(rank, world, port, out):
     dist.destroy_process_group()
 
 
-def _guarded(worker, rank, world, port, out):
+def _worker_replica_broadcast(rank, world, port, out, buffers):
+    """`buffers[q]` is rank q's full-length weight buffer, in memory every rank can address (shared memory here,
+    a peer mapping on GPUs).  Each rank's update writes its own range into every buffer; a pull is then a read
+    of the rank's own buffer after a barrier, with no gather."""
+    from oracle import reference as R
+    from workloads import generators as G, layouts
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    n_el, lam, n = 10007, 6, 2
+    w0 = G.initial_weights(layouts.flat(n_el), 5)
+    sps = ShardedParameterServer(n_el, lam, n, 0.02, 0.9, 5e-4, server_factory=ReferenceBackedServer)
+    sps.init_weights(w0)
+    sps.bind_replica_buffers(buffers)
+    whole = R.ReferencePS(n_el, lam, n, 0.02, 0.9, 5e-4, R.MOD_INV_STALENESS, 32)
+    whole.set_weights(w0.numpy())
+    ok = sps.pull_weights_from_replica() == 0 and torch.equal(buffers[rank], w0)       # filled when bound
+    kinds, learners = R.simulate_arrivals("exp", lam, 40, 9)
+    pulled, counts = {}, {}
+    for k, l in zip(kinds.tolist(), learners.tolist()):
+        if k == 0:
+            pulled[l] = sps.pull_weights()
+            whole.pull(l)
+            continue
+        b = counts.get(l, 0); counts[l] = b + 1
+        g = G.gradient(5, l, b, n_el, 1e-3)
+        whole.push(l, g.numpy())
+        if sps.push_gradient_slice(l, g[sps.lo:sps.hi].clone(), pulled[l]):
+            sps.apply_update()
+            if whole.timestamp % 4 == 0:          # a weight pull: wait, meet, read the local buffer
+                ts = sps.pull_weights_from_replica()
+                mine = buffers[rank].clone()
+                dist.barrier()                    # nobody runs ahead and overwrites while the others still compare
+                ok = ok and ts == whole.timestamp and bool(np.array_equal(mine.numpy(), whole.state()[0].astype(np.float32)))
+    ts = sps.pull_weights_from_replica()
+    ok = ok and ts == whole.timestamp == 40 // (lam // n) and bool(np.array_equal(buffers[rank].numpy(), whole.state()[0].astype(np.float32)))
+    out.put((rank, ok, sps.lo, sps.hi))
+    dist.barrier()
+    sps.destroy()
+    dist.destroy_process_group()
+
+
+def _guarded(worker, rank, world, port, out, *extra):
     """A rank that raises reports at once instead of leaving the parent to wait for its result."""
     try:
-        worker(rank, world, port, out)
+        worker(rank, world, port, out, *extra)
     except BaseException:
         out.put((rank, False, -1, -1))
         raise
 
 
-def _run_two_ranks(worker):
+def _run_two_ranks(worker, *extra):
     ctx = mp.get_context("spawn")
     out = ctx.Queue()
     port = _free_port()
-    procs = [ctx.Process(target=_guarded, args=(worker, r, 2, port, out)) for r in range(2)]
+    procs = [ctx.Process(target=_guarded, args=(worker, r, 2, port, out) + extra) for r in range(2)]
     for p in procs:
         p.start()
     got = sorted(out.get(timeout=180) for _ in procs)
@@ -233,6 +285,12 @@ def _run_two_ranks(worker):
 def test_scattered_push_needs_only_the_ranks_own_slice():
     got = _run_two_ranks(_worker_scatter)
     assert got[0][2] == 0 and got[0][3] == got[1][2] and got[1][3] == 10007
+
+
+def test_weight_broadcast_into_every_ranks_buffer_replaces_the_gather():
+    buffers = [torch.zeros(10007).share_memory_() for _ in range(2)]
+    _run_two_ranks(_worker_replica_broadcast, buffers)
+    assert torch.equal(buffers[0], buffers[1]) and float(buffers[0].abs().sum()) > 0
 
 
 def test_library_state_machine_runs_per_shard_under_gloo():

@@ -331,6 +331,32 @@ def test_exponential_penalty_shrinks_faster_than_inverse_staleness():
     assert out[R.MOD_EXP_STALENESS] == 0.5 ** 40
 
 
+def test_exponential_penalty_runs_out_through_the_denormals_to_zero():
+    """rho = 0.5 makes every scale an exact power of two, so the fp32 scale table is known in closed form all the
+    way down: 2^-tau while that is a normal or denormal fp32 number (tau <= 149), exactly zero beyond.  The
+    momentum right after such an update (m = 0, wd = 0, theta_0 = 0) is the bare product scale * g, a denormal
+    that must be kept, not flushed."""
+    ps = R.ReferencePS(4, 2, 2, 1.0, 0.0, 0.0, R.MOD_EXP_STALENESS, 32)
+    ps.set_weights(np.zeros(4, np.float32))
+    ps.pull(0); ps.pull(1)
+    g = np.array([1.0, -3.0, 0.5, 2.0 ** -3], np.float32)
+    seen = {}
+    for clock in range(160):
+        if clock in (100, 126, 127, 140, 149, 150, 155):
+            ps.push(1, g)                                   # learner 1 never pulls again: tau = clock
+            tau = int(ps.log()["tau"][-1])
+            seen[tau] = (float(ps.log()["scale"][-1]), ps.state()[1].astype(np.float32).copy())
+        ps.pull(0)
+        ps.push(0, np.zeros(4, np.float32))
+    assert sorted(seen) == [100, 127, 129, 143, 153, 155, 161]          # each stale push moved the clock on by one too
+    tiny = float(np.finfo(np.float32).tiny)                              # 2^-126
+    for tau, (scale, v) in seen.items():
+        want = np.float32(2.0 ** -tau) if tau <= 149 else np.float32(0.0)
+        assert scale == float(want) and (tau < 126 or scale < tiny)
+        assert np.array_equal(v, (np.float64(want) * g.astype(np.float64)).astype(np.float32))   # exact: powers of two
+    assert seen[143][1][0] > 0 and seen[143][1][3] > 0 and seen[153][0] == 0.0                   # denormal kept, then zero
+
+
 def _caffe_like_layers(n_el):
     b = [0, n_el // 3, n_el // 3 + 5, n_el - 7, n_el]
     return b, [1.0, 2.0, 0.5, 2.0], [1.0, 0.0, 3.0, 0.0]

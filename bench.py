@@ -330,7 +330,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     gbytes = 2 if cfg.grad_dtype == "bf16" else 4
-    fuse_t = cfg.fuse_t
+    fuse_t = args.fuse_t or cfg.fuse_t
     peak, peak_kind = hbm_peak()
 
     reps, facts, pool, ps = measure_device(P, cfg, args, dev, rank, world, local_rank, fuse_t,
@@ -668,6 +668,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="ordinary launches instead of programmatic dependent ones")
+    ap.add_argument("--fuse-t", type=int, default=0, choices=range(0, 17),
+                    help="variant: updates per kernel pass (PS_OPT_FUSE_T) instead of the workload's own; 0 = the workload's")
     ap.add_argument("--no-zigzag", action="store_true", help="every launch walks the vector forward (PS_OPT_ZIGZAG=0)")
     ap.add_argument("--bf16-mirror", action="store_true",
                     help="variant: keep a bf16 copy of the weights current in the same pass (+2 bytes per element)")
@@ -723,7 +725,7 @@ def main():
     result, e2e_detail = run_ours(args, cfg, rank, world, local_rank)
     default_run = (args.workload == "large_softsync" and not args.num_params and not args.total_params
                    and args.kernel == "auto" and not args.bf16_mirror and not args.layer_multipliers
-                   and not args.no_zigzag and not args.replicas)
+                   and not args.no_zigzag and not args.replicas and not args.fuse_t)
     if default_run and not args.no_second_config:
         result["configs"] = {"large_stale_bf16": second_config(args, rank, world, local_rank)}
     if rank == 0:

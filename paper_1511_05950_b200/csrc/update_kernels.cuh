@@ -41,8 +41,8 @@ struct LaunchParams {
     float *w;
     float *v;
     long long n;          // elements
-    float2 momentum;      // every coefficient is held twice (.x == .y): a packed multiply takes the pair as ONE
-                          // 64-bit operand straight from parameter space instead of building it with two moves
+    float2 momentum;      // every coefficient is held twice (.x == .y), so that a packed multiply can take the
+                          // pair as ONE 64-bit operand straight from parameter space
     int T;                // groups in this pass
     int c;                // gradients per group
     int overlap;          // 1: launched as a programmatic dependent; gradients may be fetched early
